@@ -1,0 +1,161 @@
+/*
+ * liblaq -- the eviction step of Lookahead Q-Cache (LAQ) on one NVIDIA B200 (sm_100a).
+ *
+ * Given the full prompt key/value cache of every layer and a small window of post-RoPE
+ * "lookahead" queries (the Q-Cache of Section 4.2), the library ranks every cached prompt
+ * position and keeps a fixed budget of them per KV head (Section 4.3, Eq. 4):
+ *
+ *     M_ahead = ArgSort( sum_{q_i in Q} q_i K^T )[:B]
+ *
+ * Notation (used in every comment of this library):
+ *   NL, Bt      layers, batch
+ *   Hq, Hkv     query heads, KV heads;  G = Hq / Hkv  query heads share one KV head
+ *   D           head dimension (128)
+ *   L           prompt length = cached positions before eviction
+ *   W           lookahead queries per query head (the observation window)
+ *   R           retained tail: the last R prompt positions are always kept
+ *   k           1-D pooling kernel (odd)
+ *   B           budget: positions kept per (layer, batch, KV head), tail included
+ *   unit        one (layer, batch, KV head) triple; U = NL*Bt*Hkv units, all independent
+ *   M = G*W     softmax rows of a unit;  Ls = L-R scored positions;  Kb = B-R selected slots
+ *
+ * What one unit computes (Eq. 4 read as attention weights; the paper's Eq. 4 omits the scale,
+ * the softmax, the GQA reduction and the pooling, which follow the SnapKV-style "standard KV
+ * cache eviction" the paper builds on, Sections 1 and 5.1):
+ *   1. logits   s[r][j] = scale * <q_r, k_j>,  r = g*W+i over the G heads x W queries, j in [0,L)
+ *   2. softmax  P[r][j] = exp(s[r][j]-m_r) / l_r,  m_r = max_j s[r][j],  l_r = sum_j exp(s[r][j]-m_r)
+ *   3. column sums  c[j] = sum_r P[r][j]
+ *   4. pooling  p[j] = (1/k) * sum_{|t|<=k/2, 0<=j+t<Ls} c[j+t],  j in [0,Ls)   (zero padded)
+ *   5. top-k    the Kb positions of largest p (ties: lower position wins), written ascending,
+ *               followed by the tail Ls..L-1
+ *   6. gather   K_out[t] = K[idx[t]],  V_out[t] = V[idx[t]]
+ *
+ * Conventions common to every entry point
+ *   - Every data pointer is a DEVICE pointer owned by the caller. Nothing is allocated, retained
+ *     or freed by the library; scratch memory is the caller's workspace `ws` of at least
+ *     laq_workspace_bytes() bytes, 256-byte aligned. A workspace may be reused by later calls on
+ *     the same stream; two calls that overlap on the GPU need two workspaces.
+ *   - Q, K, V, K_out, V_out hold bf16; the innermost (head_dim) stride is 1 and every other
+ *     stride, given in ELEMENTS in laq_params, is a multiple of 8 (16 bytes). Base pointers are
+ *     16-byte aligned.
+ *   - Calls validate on the host, enqueue kernels on `cuda_stream` (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream) and return without synchronising. A non-OK status
+ *     means nothing was enqueued, except LAQ_ERR_CUDA from a failed launch.
+ *   - Device-side waits are bounded. If one runs out the kernel records it in the workspace and
+ *     finishes; laq_last_device_status() reads that record back (it synchronises the stream).
+ *   - No exceptions cross the boundary; the library keeps no global mutable state apart from
+ *     cached per-device attributes.
+ */
+#ifndef LAQ_H_
+#define LAQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LAQ_OK = 0,
+  LAQ_ERR_INVALID_ARG = 1, /* null pointer, bad size relation, misaligned pointer or stride */
+  LAQ_ERR_UNSUPPORTED = 2, /* a valid problem this build has no kernel for (e.g. head_dim != 128) */
+  LAQ_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or smaller than laq_workspace_bytes() */
+  LAQ_ERR_CUDA = 4,        /* a CUDA runtime or driver call failed */
+  LAQ_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out (see laq_last_device_status) */
+  LAQ_ERR_INTERNAL = 6
+} laq_status;
+
+typedef enum { LAQ_POOL_AVG = 0 } laq_pool_mode;
+
+/* Problem description. Plain data; copy freely. All strides are in bf16 ELEMENTS. */
+typedef struct {
+  int32_t n_layers;    /* NL >= 1 */
+  int32_t batch;       /* Bt >= 1 */
+  int32_t n_q_heads;   /* Hq, a multiple of n_kv_heads */
+  int32_t n_kv_heads;  /* Hkv >= 1; query head h reads KV head h / G */
+  int32_t head_dim;    /* D; 128 is the supported value */
+  int32_t prompt_len;  /* L */
+  int32_t window_len;  /* W >= 1 lookahead queries per query head; G*W <= 256 */
+  int32_t keep_tail;   /* R, 0 <= R < B: last R positions always kept and never scored */
+  int32_t pool_kernel; /* k, odd >= 1; 1 disables pooling */
+  int32_t pool_mode;   /* laq_pool_mode */
+  int32_t budget;      /* B, R < B < L */
+  float softmax_scale; /* 0 selects 1/sqrt(head_dim) */
+  /* Q [NL][Bt][Hq][W][D] */
+  int64_t q_stride_layer, q_stride_batch, q_stride_head, q_stride_pos;
+  /* K [NL][Bt][Hkv][L][D] */
+  int64_t k_stride_layer, k_stride_batch, k_stride_head, k_stride_pos;
+  /* V [NL][Bt][Hkv][L][D] */
+  int64_t v_stride_layer, v_stride_batch, v_stride_head, v_stride_pos;
+  /* K_out and V_out [NL][Bt][Hkv][B][D] (the same strides serve both) */
+  int64_t o_stride_layer, o_stride_batch, o_stride_head, o_stride_pos;
+} laq_params;
+
+/* Fills the stride fields of `p` for densely packed tensors in the index order shown above. */
+void laq_params_dense_strides(laq_params* p);
+
+/* Bytes of caller-provided device scratch that laq_score / laq_evict need for `p`
+ * (0 if `p` is invalid). laq_select and laq_compact need none. */
+size_t laq_workspace_bytes(const laq_params* p);
+
+/*
+ * Steps 1-4 (Eq. 4's sum over the window, Section 4.3): pooled importance of every scored
+ * position.
+ *   q       device, bf16, lookahead queries, layout/strides from `p`
+ *   k       device, bf16, prompt keys
+ *   scores  device, fp32, dense [NL][Bt][Hkv][L-R]; written in full
+ *   ws      device scratch, ws_bytes >= laq_workspace_bytes(p)
+ * Errors: LAQ_ERR_INVALID_ARG, LAQ_ERR_UNSUPPORTED, LAQ_ERR_WORKSPACE, LAQ_ERR_CUDA.
+ */
+laq_status laq_score(const laq_params* p, const void* q, const void* k, float* scores,
+                     void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Step 5 (Eq. 4's ArgSort(...)[:B]): per unit, the B-R positions of largest score, ties to the
+ * lower position, then the retained tail.
+ *   scores  device, fp32, dense [NL][Bt][Hkv][L-R], every value >= 0 and not NaN
+ *   idx     device, int32, dense [NL][Bt][Hkv][B]; first B-R entries strictly ascending in
+ *           [0, L-R), last R entries are L-R .. L-1
+ * Only n_layers, batch, n_kv_heads, prompt_len, keep_tail and budget of `p` are read.
+ */
+laq_status laq_select(const laq_params* p, const float* scores, int32_t* idx, void* cuda_stream);
+
+/*
+ * Step 6 ("cache re-eviction based on the given budget", Section 4.3): gathers the kept rows.
+ *   k, v          device, bf16, prompt keys and values
+ *   idx           device, int32, dense [NL][Bt][Hkv][B], every entry in [0, L)
+ *   k_out, v_out  device, bf16, [NL][Bt][Hkv][B][D] with the o_stride_* strides; either may be
+ *                 NULL to skip that tensor. Must not overlap k / v.
+ */
+laq_status laq_compact(const laq_params* p, const void* k, const void* v, const int32_t* idx,
+                       void* k_out, void* v_out, void* cuda_stream);
+
+/*
+ * Steps 1-6 in one call (the whole re-eviction of Section 4.3 for all layers and heads).
+ *   idx     optional (NULL allowed) device int32 [NL][Bt][Hkv][B]: receives the kept positions
+ *   scores  optional (NULL allowed) device fp32 [NL][Bt][Hkv][L-R]: receives the pooled scores
+ * Other arguments as in laq_score / laq_compact.
+ */
+laq_status laq_evict(const laq_params* p, const void* q, const void* k, const void* v,
+                     void* k_out, void* v_out, int32_t* idx, float* scores, void* ws,
+                     size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Synchronises `cuda_stream` and reports what the last laq_score / laq_evict call that used
+ * `ws` recorded on the device: LAQ_OK, LAQ_ERR_TIMEOUT (a bounded wait ran out; outputs are
+ * not valid) or LAQ_ERR_CUDA (the synchronise or the read-back failed).
+ */
+laq_status laq_last_device_status(const laq_params* p, const void* ws, size_t ws_bytes,
+                                  void* cuda_stream);
+
+/* Kernel launches the most recent call on this host thread enqueued (for accounting). */
+int laq_last_launch_count(void);
+
+const char* laq_status_string(laq_status s);
+int laq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LAQ_H_ */

@@ -1,0 +1,205 @@
+/*
+ * CPU oracle for the Lookahead Q-Cache (LAQ) re-eviction step -- TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, fp64 statement of what Section 4.3 (Eq. 4) computes, with the steps the
+ * equation leaves implicit (scale, softmax, GQA sum, average pooling, retained tail) taken from
+ * the "standard KV cache eviction" the paper builds on (Sections 1 and 5.1, SnapKV's average
+ * pooling). It shares no code with the CUDA library and must never be called from it: only the
+ * tests, the smoke check and the benchmark's cpu_baseline leg may use this file.
+ *
+ * Inputs are bf16 bit patterns (uint16_t), converted exactly to double. Every loop is the
+ * definition written out; there is no blocking, fusion or reordering. OpenMP is used only
+ * across independent (layer, batch, KV head) units in laq_oracle_evict.
+ *
+ * Pins (tests/test_oracle_pins.py): brute-force softmax on tiny inputs, torch.softmax /
+ * torch.topk in fp64 as independent library routines, row sums = 1, sum of column sums = M,
+ * identical-key closed forms for pooling and tie-break, key-shift invariance, additivity over
+ * heads and queries, budget nestedness, planted key kept.
+ * Parity unpinned by the paper: the softmax reading of Eq. 4, the sum over the GQA group, the
+ * average pool with zero padding and divisor k, and the retained tail are conventions fixed by
+ * the benchmark spec, not by a value the paper prints.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static double bf16_to_double(uint16_t h) {
+  uint32_t u = ((uint32_t)h) << 16;
+  float f;
+  memcpy(&f, &u, sizeof f);
+  return (double)f;
+}
+
+/*
+ * Steps 1-3 of the unit computation (Eq. 4, "sum_{q_i in Q} q_i K^T", read as attention
+ * weights): logits, per-row softmax over all L keys, column sums over the G*W rows.
+ *   q        [G][W][D] bf16, the lookahead queries of the G query heads that share this KV head
+ *   k        [L][D]    bf16, prompt keys of this KV head
+ *   c        [L]       out: c[j] = sum_r P[r][j]
+ *   row_max  [G*W]     out (may be NULL): m_r
+ *   row_sum  [G*W]     out (may be NULL): l_r
+ */
+void laq_oracle_unit_colsum(const uint16_t* q, const uint16_t* k, int G, int W, int D, int L,
+                            double scale, double* c, double* row_max, double* row_sum) {
+  const int M = G * W;
+  double* s = (double*)malloc((size_t)L * sizeof(double));
+  for (int j = 0; j < L; ++j) c[j] = 0.0;
+  for (int r = 0; r < M; ++r) {
+    /* logits of row r against every key (Eq. 4: q_i K^T, scaled) */
+    for (int j = 0; j < L; ++j) {
+      double acc = 0.0;
+      for (int d = 0; d < D; ++d)
+        acc += bf16_to_double(q[(size_t)r * D + d]) * bf16_to_double(k[(size_t)j * D + d]);
+      s[j] = scale * acc;
+    }
+    /* softmax over the L prompt keys */
+    double m = s[0];
+    for (int j = 1; j < L; ++j)
+      if (s[j] > m) m = s[j];
+    double l = 0.0;
+    for (int j = 0; j < L; ++j) l += exp(s[j] - m);
+    /* Eq. 4's sum over the window (and over the heads of the group) */
+    for (int j = 0; j < L; ++j) c[j] += exp(s[j] - m) / l;
+    if (row_max) row_max[r] = m;
+    if (row_sum) row_sum[r] = l;
+  }
+  free(s);
+}
+
+/*
+ * Step 4: average pooling over the scored positions [0, Ls), stride 1, zero padding of k/2 on
+ * both sides, divisor always k (SnapKV-style pooling, Section 5.1 "employs average pooling").
+ */
+void laq_oracle_pool(const double* c, int Ls, int kernel, double* p) {
+  const int h = kernel / 2;
+  for (int j = 0; j < Ls; ++j) {
+    double acc = 0.0;
+    for (int t = -h; t <= h; ++t) {
+      const int jj = j + t;
+      if (jj >= 0 && jj < Ls) acc += c[jj];
+    }
+    p[j] = acc / (double)kernel;
+  }
+}
+
+/*
+ * Step 5 (Eq. 4's ArgSort(...)[:B], descending): the Kb = B-R positions of largest p, a tie
+ * going to the lower position; written ascending and followed by the tail Ls..L-1.
+ * Selection by repeated scan for the best remaining position: O(Ls*Kb), obviously correct.
+ */
+void laq_oracle_select(const double* p, int L, int R, int B, int32_t* idx) {
+  const int Ls = L - R, Kb = B - R;
+  unsigned char* taken = (unsigned char*)calloc((size_t)(Ls > 0 ? Ls : 1), 1);
+  for (int n = 0; n < Kb; ++n) {
+    int best = -1;
+    for (int j = 0; j < Ls; ++j) {
+      if (taken[j]) continue;
+      if (best < 0 || p[j] > p[best]) best = j; /* strict '>' keeps the lower position on ties */
+    }
+    taken[best] = 1;
+  }
+  int t = 0;
+  for (int j = 0; j < Ls; ++j)
+    if (taken[j]) idx[t++] = j;
+  for (int j = Ls; j < L; ++j) idx[t++] = j;
+  free(taken);
+}
+
+/* Same selection in O(Ls log Ls) for the timed baseline and large parity samples: sort positions
+ * by (p descending, position ascending), keep the first Kb. Checked against laq_oracle_select. */
+typedef struct {
+  double p;
+  int32_t j;
+} laq_oracle_pair;
+
+static int pair_cmp(const void* a, const void* b) {
+  const laq_oracle_pair* x = (const laq_oracle_pair*)a;
+  const laq_oracle_pair* y = (const laq_oracle_pair*)b;
+  if (x->p > y->p) return -1;
+  if (x->p < y->p) return 1;
+  return (x->j > y->j) - (x->j < y->j);
+}
+
+static int int_cmp(const void* a, const void* b) {
+  const int32_t x = *(const int32_t*)a, y = *(const int32_t*)b;
+  return (x > y) - (x < y);
+}
+
+void laq_oracle_select_sorted(const double* p, int L, int R, int B, int32_t* idx) {
+  const int Ls = L - R, Kb = B - R;
+  laq_oracle_pair* a = (laq_oracle_pair*)malloc((size_t)(Ls > 0 ? Ls : 1) * sizeof *a);
+  for (int j = 0; j < Ls; ++j) {
+    a[j].p = p[j];
+    a[j].j = j;
+  }
+  qsort(a, (size_t)Ls, sizeof *a, pair_cmp);
+  for (int t = 0; t < Kb; ++t) idx[t] = a[t].j;
+  qsort(idx, (size_t)Kb, sizeof *idx, int_cmp);
+  for (int j = Ls; j < L; ++j) idx[Kb + (j - Ls)] = j;
+  free(a);
+}
+
+/* Step 6: bit copies of the kept rows. src [L][D], dst [B][D], bf16 bit patterns. */
+void laq_oracle_compact(const uint16_t* src, const int32_t* idx, int B, int D, uint16_t* dst) {
+  for (int t = 0; t < B; ++t)
+    for (int d = 0; d < D; ++d) dst[(size_t)t * D + d] = src[(size_t)idx[t] * D + d];
+}
+
+/*
+ * The whole step for densely packed tensors:
+ *   Q [NL][Bt][Hq][W][D], K and V [NL][Bt][Hkv][L][D]  (bf16 bit patterns)
+ *   scores [NL][Bt][Hkv][L-R] pooled (may be NULL), colsum [NL][Bt][Hkv][L] (may be NULL),
+ *   idx [NL][Bt][Hkv][B] (may be NULL; then k_out/v_out are not written),
+ *   k_out, v_out [NL][Bt][Hkv][B][D] (may be NULL).
+ * `unit_list` (may be NULL) restricts the work to n_units listed unit numbers
+ * u = (layer*Bt + b)*Hkv + h; outputs of other units are left untouched.
+ * Query head h*G+g belongs to KV head h. Returns the number of OpenMP threads used.
+ */
+int laq_oracle_evict(const uint16_t* q, const uint16_t* k, const uint16_t* v, int NL, int Bt,
+                     int Hq, int Hkv, int D, int L, int W, int R, int kernel, int B,
+                     double scale, const int64_t* unit_list, int64_t n_units, double* scores,
+                     double* colsum, int32_t* idx, uint16_t* k_out, uint16_t* v_out,
+                     int fast_select) {
+  const int G = Hq / Hkv;
+  const int Ls = L - R;
+  const int64_t U = (int64_t)NL * Bt * Hkv;
+  const int64_t n = unit_list ? n_units : U;
+  int threads = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+  {
+#pragma omp single
+    threads = omp_get_num_threads();
+  }
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+  for (int64_t t = 0; t < n; ++t) {
+    const int64_t u = unit_list ? unit_list[t] : t;
+    const int64_t h = u % Hkv;
+    const int64_t lb = u / Hkv; /* layer*Bt + b */
+    const uint16_t* qu = q + ((lb * Hq + h * G) * (int64_t)W) * D;
+    const uint16_t* ku = k + u * (int64_t)L * D;
+    double* c = (double*)malloc((size_t)L * sizeof(double));
+    double* p = (double*)malloc((size_t)(Ls > 0 ? Ls : 1) * sizeof(double));
+    laq_oracle_unit_colsum(qu, ku, G, W, D, L, scale, c, NULL, NULL);
+    laq_oracle_pool(c, Ls, kernel, p);
+    if (colsum) memcpy(colsum + u * (int64_t)L, c, (size_t)L * sizeof(double));
+    if (scores) memcpy(scores + u * (int64_t)Ls, p, (size_t)Ls * sizeof(double));
+    if (idx) {
+      int32_t* iu = idx + u * (int64_t)B;
+      if (fast_select)
+        laq_oracle_select_sorted(p, L, R, B, iu);
+      else
+        laq_oracle_select(p, L, R, B, iu);
+      if (k_out) laq_oracle_compact(ku, iu, B, D, k_out + u * (int64_t)B * D);
+      if (v_out) laq_oracle_compact(v + u * (int64_t)L * D, iu, B, D, v_out + u * (int64_t)B * D);
+    }
+    free(c);
+    free(p);
+  }
+  return threads;
+}

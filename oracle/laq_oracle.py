@@ -1,0 +1,135 @@
+"""ctypes access to the fp64 CPU oracle (``laq_oracle.c``) -- TEST INFRASTRUCTURE ONLY.
+
+The oracle states what Section 4.3 (Eq. 4) computes in plain loops; this module only compiles it
+with gcc, marshals numpy arrays and holds no arithmetic of the method. It shares nothing with the
+CUDA library and is imported only by the tests, the smoke check and the benchmark's CPU baseline.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "laq_oracle.c")
+_LIB = os.path.join(_HERE, "liblaq_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compiles the oracle with gcc (-O2, OpenMP over units) if the library is missing or stale."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True, cwd=_HERE)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        vp, i, d, i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_double, ctypes.c_int64
+        lib.laq_oracle_unit_colsum.argtypes = [vp, vp, i, i, i, i, d, vp, vp, vp]
+        lib.laq_oracle_unit_colsum.restype = None
+        lib.laq_oracle_pool.argtypes = [vp, i, i, vp]
+        lib.laq_oracle_pool.restype = None
+        lib.laq_oracle_select.argtypes = [vp, i, i, i, vp]
+        lib.laq_oracle_select.restype = None
+        lib.laq_oracle_select_sorted.argtypes = [vp, i, i, i, vp]
+        lib.laq_oracle_select_sorted.restype = None
+        lib.laq_oracle_compact.argtypes = [vp, vp, i, i, vp]
+        lib.laq_oracle_compact.restype = None
+        lib.laq_oracle_evict.argtypes = [vp, vp, vp, i, i, i, i, i, i, i, i, i, i, d, vp, i64,
+                                         vp, vp, vp, vp, vp, i]
+        lib.laq_oracle_evict.restype = i
+        _lib = lib
+    return _lib
+
+
+def _bits(a) -> np.ndarray:
+    """bf16 bit patterns as a C-contiguous uint16 array (accepts uint16 numpy or a bf16 CPU tensor)."""
+    if not isinstance(a, np.ndarray):  # torch tensor, bf16 or int16/uint16 view
+        import torch
+
+        a = a.detach().cpu().contiguous()
+        if a.dtype == torch.bfloat16:
+            a = a.view(torch.int16)
+        a = a.numpy()
+    return np.ascontiguousarray(a).view(np.uint16)
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def unit_colsum(q, k, scale=None):
+    """q [G][W][D], k [L][D] bf16 -> (c [L], row_max [G*W], row_sum [G*W]) in fp64."""
+    q, k = _bits(q), _bits(k)
+    G, W, D = q.shape
+    L = k.shape[0]
+    assert k.shape[1] == D
+    scale = 1.0 / np.sqrt(D) if scale is None else float(scale)
+    c = np.empty(L, np.float64)
+    m = np.empty(G * W, np.float64)
+    l = np.empty(G * W, np.float64)
+    _load().laq_oracle_unit_colsum(_ptr(q), _ptr(k), G, W, D, L, scale, _ptr(c), _ptr(m), _ptr(l))
+    return c, m, l
+
+
+def pool(c, Ls, kernel):
+    c = np.ascontiguousarray(c, np.float64)
+    assert c.shape[0] >= Ls
+    p = np.empty(Ls, np.float64)
+    _load().laq_oracle_pool(_ptr(c), Ls, kernel, _ptr(p))
+    return p
+
+
+def select(p, L, R, B, sorted_variant=False):
+    """p [L-R] scores (any float dtype, promoted exactly to fp64) -> idx [B] int32."""
+    p = np.ascontiguousarray(p, np.float64)
+    assert p.shape[0] == L - R and 0 <= R < B <= L
+    idx = np.empty(B, np.int32)
+    fn = _load().laq_oracle_select_sorted if sorted_variant else _load().laq_oracle_select
+    fn(_ptr(p), L, R, B, _ptr(idx))
+    return idx
+
+
+def compact(src, idx):
+    src = _bits(src)
+    idx = np.ascontiguousarray(idx, np.int32)
+    dst = np.empty((idx.shape[0], src.shape[1]), np.uint16)
+    _load().laq_oracle_compact(_ptr(src), _ptr(idx), idx.shape[0], src.shape[1], _ptr(dst))
+    return dst
+
+
+def evict(q, k, v, R, kernel, B, scale=None, units=None, want_colsum=False, fast_select=True,
+          want_idx=True):
+    """Whole step on dense tensors. q [NL][Bt][Hq][W][D], k/v [NL][Bt][Hkv][L][D] (bf16).
+
+    Returns a dict with 'scores' [NL,Bt,Hkv,L-R] fp64, 'idx' [NL,Bt,Hkv,B] int32, 'k_out',
+    'v_out' [NL,Bt,Hkv,B,D] uint16 bit patterns, 'threads', and 'colsum' if asked. With `units`
+    (unit numbers (layer*Bt+b)*Hkv+h) only those units are computed; the rest stays zero.
+    """
+    q, k = _bits(q), _bits(k)
+    v = None if v is None else _bits(v)
+    NL, Bt, Hq, W, D = q.shape
+    Hkv, L = k.shape[2], k.shape[3]
+    assert k.shape == (NL, Bt, Hkv, L, D) and Hq % Hkv == 0
+    scale = 1.0 / np.sqrt(D) if scale is None else float(scale)
+    Ls = L - R
+    scores = np.zeros((NL, Bt, Hkv, Ls), np.float64)
+    colsum = np.zeros((NL, Bt, Hkv, L), np.float64) if want_colsum else None
+    idx = np.zeros((NL, Bt, Hkv, B), np.int32) if want_idx else None
+    k_out = np.zeros((NL, Bt, Hkv, B, D), np.uint16) if want_idx else None
+    v_out = np.zeros((NL, Bt, Hkv, B, D), np.uint16) if (want_idx and v is not None) else None
+    ul = None if units is None else np.ascontiguousarray(units, np.int64)
+    threads = _load().laq_oracle_evict(
+        _ptr(q), _ptr(k), _ptr(v), NL, Bt, Hq, Hkv, D, L, W, R, kernel, B, scale, _ptr(ul),
+        0 if ul is None else ul.shape[0], _ptr(scores), _ptr(colsum), _ptr(idx), _ptr(k_out),
+        _ptr(v_out), 1 if fast_select else 0)
+    out = {"scores": scores, "idx": idx, "k_out": k_out, "v_out": v_out, "threads": threads}
+    if want_colsum:
+        out["colsum"] = colsum
+    return out

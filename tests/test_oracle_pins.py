@@ -1,0 +1,298 @@
+"""Pins for the fp64 CPU oracle: each test checks it against something other than itself -- a
+hand-derived example, brute force, an independent library routine (torch fp64 on CPU), a closed
+form or an invariant -- chosen so that a dropped term, a wrong sign or index or a transposed
+operand fails at least one of them. No GPU needed."""
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import laq_oracle as orc
+from paper_2505_20334_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bf16(t):
+    return t.to(torch.bfloat16)
+
+
+def rand_bf16(shape, seed, scale=1.0):
+    g = torch.Generator().manual_seed(seed)
+    return bf16(torch.randn(shape, generator=g) * scale)
+
+
+def torch_colsum(q, k, scale):
+    """Independent statement with library routines: softmax over keys, summed over rows."""
+    G, W, D = q.shape
+    s = (q.double().reshape(G * W, D) @ k.double().T) * scale
+    return torch.softmax(s, dim=-1).sum(0).numpy(), s
+
+
+# ---------------------------------------------------------------- hand-derived example
+def test_hand_example_exact_rationals():
+    vals = {}
+    with open(os.path.join(GOLDEN, "hand_example.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            key, *nums = line.split()
+            vals[key] = [int(x) for x in nums]
+    q = bf16(torch.tensor([[[1.0], [2.0]]]))  # G=1, W=2, D=1
+    k = bf16(torch.tensor([[0.0], [1.0], [2.0]]))
+    c, m, l = orc.unit_colsum(q, k, scale=math.log(2.0))
+    want_c = [Fraction(n, vals["c_den"][0]) for n in vals["c_num"]]
+    np.testing.assert_allclose(c, [float(x) for x in want_c], rtol=1e-14)
+    np.testing.assert_allclose(m, [2 * math.log(2), 4 * math.log(2)], rtol=1e-15)
+    want_l = [Fraction(n, d) for n, d in zip(vals["l_num"], vals["l_den"])]
+    np.testing.assert_allclose(l, [float(x) for x in want_l], rtol=1e-14)
+    p = orc.pool(c, 3, 3)
+    want_p = [Fraction(n, vals["p_den"][0]) for n in vals["p_num"]]
+    np.testing.assert_allclose(p, [float(x) for x in want_p], rtol=1e-14)
+    idx = orc.select(p, L=3, R=0, B=2)
+    assert idx.tolist() == [1, 2]
+
+
+# ---------------------------------------------------------------- softmax / column sums
+@pytest.mark.parametrize("G,W,D,L", [(1, 1, 2, 3), (2, 3, 4, 7), (3, 2, 8, 16)])
+def test_bruteforce_softmax_tiny(G, W, D, L):
+    q = rand_bf16((G, W, D), 1)
+    k = rand_bf16((L, D), 2)
+    scale = 1.0 / math.sqrt(D)
+    c, m, l = orc.unit_colsum(q, k)
+    ql = q.double().reshape(G * W, D).tolist()
+    kl = k.double().tolist()
+    want = [0.0] * L
+    for r in range(G * W):
+        e = [math.exp(scale * sum(ql[r][d] * kl[j][d] for d in range(D))) for j in range(L)]
+        z = math.fsum(e)  # naive exp / sum(exp): no max subtraction
+        for j in range(L):
+            want[j] += e[j] / z
+        smax = max(scale * sum(ql[r][d] * kl[j][d] for d in range(D)) for j in range(L))
+        assert m[r] == pytest.approx(smax, rel=1e-14, abs=1e-15)
+        assert m[r] + math.log(l[r]) == pytest.approx(math.log(z), rel=1e-13, abs=1e-13)
+    np.testing.assert_allclose(c, want, rtol=1e-13)
+
+
+@pytest.mark.parametrize("G,W,D,L,seed", [(4, 8, 128, 300, 3), (1, 5, 64, 77, 4), (8, 2, 32, 129, 5)])
+def test_against_torch_softmax_fp64(G, W, D, L, seed):
+    q = rand_bf16((G, W, D), seed)
+    k = rand_bf16((L, D), seed + 100, scale=1.5)
+    scale = 1.0 / math.sqrt(D)
+    c, m, l = orc.unit_colsum(q, k)
+    want, s = torch_colsum(q, k, scale)
+    np.testing.assert_allclose(c, want, rtol=1e-12, atol=1e-300)
+    np.testing.assert_allclose(m, s.max(dim=-1).values.numpy(), rtol=1e-14)
+    np.testing.assert_allclose(m + np.log(l), torch.logsumexp(s, dim=-1).numpy(), rtol=1e-13)
+    # each query's probabilities sum to one, so the column sums add up to M = G*W
+    assert c.sum() == pytest.approx(G * W, rel=1e-12)
+    assert (c > 0).all()
+
+
+def test_explicit_scale_argument_is_used():
+    q = rand_bf16((2, 2, 16), 11)
+    k = rand_bf16((40, 16), 12)
+    c, _, _ = orc.unit_colsum(q, k, scale=0.37)
+    want, _ = torch_colsum(q, k, 0.37)
+    np.testing.assert_allclose(c, want, rtol=1e-12)
+    c0, _, _ = orc.unit_colsum(q, k)
+    assert not np.allclose(c, c0, rtol=1e-3)
+
+
+def test_zero_queries_give_uniform_attention():
+    G, W, D, L = 2, 3, 16, 50
+    q = bf16(torch.zeros((G, W, D)))
+    k = rand_bf16((L, D), 7)
+    c, m, l = orc.unit_colsum(q, k)
+    np.testing.assert_allclose(c, np.full(L, G * W / L), rtol=1e-14)
+    np.testing.assert_allclose(l, np.full(G * W, L), rtol=1e-14)
+
+
+def test_key_shift_invariance_exact_inputs():
+    # integers are exact in bf16, so shifting every key by the same vector changes each row's
+    # logits by a constant and leaves the softmax untouched
+    g = torch.Generator().manual_seed(21)
+    q = bf16(torch.randint(-2, 3, (2, 2, 8), generator=g).float())
+    k = torch.randint(-4, 5, (33, 8), generator=g).float()
+    delta = torch.randint(-3, 4, (8,), generator=g).float()
+    c1, _, _ = orc.unit_colsum(q, bf16(k))
+    c2, _, _ = orc.unit_colsum(q, bf16(k + delta))
+    np.testing.assert_allclose(c1, c2, rtol=1e-12)
+
+
+def test_additivity_over_heads_and_queries():
+    G, W, D, L = 3, 4, 32, 90
+    q = rand_bf16((G, W, D), 31)
+    k = rand_bf16((L, D), 32)
+    c, _, _ = orc.unit_colsum(q, k)
+    by_head = sum(orc.unit_colsum(q[g:g + 1], k)[0] for g in range(G))
+    by_query = sum(orc.unit_colsum(q[:, i:i + 1], k)[0] for i in range(W))
+    np.testing.assert_allclose(c, by_head, rtol=1e-12)
+    np.testing.assert_allclose(c, by_query, rtol=1e-12)
+
+
+# ---------------------------------------------------------------- pooling
+@pytest.mark.parametrize("kernel", [1, 3, 5, 7])
+def test_pool_matches_library_avg_pool(kernel):
+    g = torch.Generator().manual_seed(41)
+    c = torch.rand(57, generator=g, dtype=torch.float64)
+    p = orc.pool(c.numpy(), 57, kernel)
+    want = torch.nn.functional.avg_pool1d(c[None, None], kernel, stride=1, padding=kernel // 2,
+                                          count_include_pad=True)[0, 0].numpy()
+    np.testing.assert_allclose(p, want, rtol=1e-13)
+    if kernel == 1:
+        assert (p == c.numpy()).all()
+
+
+def test_pool_ignores_tail_positions():
+    # positions >= Ls (the retained tail) are invisible to the pool
+    c = np.arange(1.0, 21.0)
+    p_a = orc.pool(c, 15, 5)
+    c2 = c.copy()
+    c2[15:] = 1e9
+    p_b = orc.pool(c2, 15, 5)
+    assert (p_a == p_b).all()
+    assert p_a[14] == pytest.approx((13 + 14 + 15) / 5.0)
+
+
+def test_pool_closed_forms():
+    kernel, Ls, val = 7, 40, 0.125
+    p = orc.pool(np.full(Ls, val), Ls, kernel)
+    h = kernel // 2
+    for j in range(Ls):
+        cover = min(j, h) + 1 + min(Ls - 1 - j, h)
+        assert p[j] == pytest.approx(val * cover / kernel, rel=1e-15)
+    c = np.random.default_rng(5).random(Ls)
+    p = orc.pool(c, Ls, kernel)
+    cover = np.array([min(j, h) + 1 + min(Ls - 1 - j, h) for j in range(Ls)])
+    assert p.sum() == pytest.approx((c * cover).sum() / kernel, rel=1e-13)
+
+
+# ---------------------------------------------------------------- selection
+def test_select_identical_keys_closed_form():
+    # identical keys: c_j = M/L everywhere, so only the pool's edge attenuation and the tie-break
+    # decide: the kept set is [k/2, k/2 + Kb) followed by the tail
+    G, W, D, L, R, kernel, B = 2, 4, 16, 64, 4, 7, 20
+    q = rand_bf16((1, 1, G, W, D), 51)
+    k = bf16(torch.ones((1, 1, 1, L, D)) * 0.5)
+    out = orc.evict(q, k, k, R, kernel, B, fast_select=False)
+    want = list(range(kernel // 2, kernel // 2 + (B - R))) + list(range(L - R, L))
+    assert out["idx"][0, 0, 0].tolist() == want
+    out2 = orc.evict(q, k, k, R, kernel, B, fast_select=True)
+    assert out2["idx"][0, 0, 0].tolist() == want
+    np.testing.assert_allclose(out["scores"][0, 0, 0, 10], G * W / L, rtol=1e-13)
+
+
+def test_select_reduces_to_topk_of_raw_logits():
+    # W = G = k = 1, R = 0: softmax is monotone, so the kept set is the top-B of q.k
+    D, L, B = 32, 200, 17
+    q = rand_bf16((1, 1, 1, 1, D), 61)
+    k = rand_bf16((1, 1, 1, L, D), 62)
+    out = orc.evict(q, k, k, 0, 1, B)
+    logits = k[0, 0, 0].double() @ q[0, 0, 0, 0].double()
+    want = sorted(torch.topk(logits, B).indices.tolist())
+    assert out["idx"][0, 0, 0].tolist() == want
+
+
+def test_select_structure_ties_and_variants_agree():
+    rng = np.random.default_rng(71)
+    for L, R, B in [(50, 4, 12), (33, 0, 33), (40, 8, 9), (17, 3, 16)]:
+        p = rng.integers(0, 6, L - R).astype(np.float64)  # many ties
+        a = orc.select(p, L, R, B)
+        b = orc.select(p, L, R, B, sorted_variant=True)
+        assert (a == b).all()
+        Kb = B - R
+        assert a.shape == (B,) and len(set(a.tolist())) == B
+        assert (np.diff(a[:Kb]) > 0).all() and (a[:Kb] < L - R).all() if Kb > 1 else True
+        assert a[Kb:].tolist() == list(range(L - R, L))
+        # independent statement: stable argsort of -p (ties keep the lower position first)
+        want = np.sort(np.argsort(-p, kind="stable")[:Kb])
+        assert (a[:Kb] == want).all()
+        thr = np.sort(p)[::-1][Kb - 1]
+        assert (p[a[:Kb]] >= thr).all()
+
+
+def test_select_budget_nestedness():
+    p = np.random.default_rng(81).random(300)
+    prev = set()
+    for B in [8, 16, 64, 200]:
+        cur = set(orc.select(p, 304, 4, B).tolist())
+        assert prev <= cur
+        prev = cur
+
+
+# ---------------------------------------------------------------- compaction, GQA mapping, whole step
+def test_compact_is_row_gather():
+    src = rand_bf16((30, 16), 91)
+    idx = np.array([3, 4, 9, 29, 0], np.int32)
+    got = orc.compact(src, idx)
+    want = src.view(torch.int16).numpy().view(np.uint16)[idx]
+    assert (got == want).all()
+
+
+def test_evict_gqa_mapping_and_dense_layout():
+    NL, Bt, Hq, Hkv, D, L, W, R, kernel, B = 2, 2, 6, 2, 16, 48, 3, 3, 3, 11
+    G = Hq // Hkv
+    q = rand_bf16((NL, Bt, Hq, W, D), 101)
+    k = rand_bf16((NL, Bt, Hkv, L, D), 102)
+    v = rand_bf16((NL, Bt, Hkv, L, D), 103)
+    out = orc.evict(q, k, v, R, kernel, B, want_colsum=True, fast_select=False)
+    # library statement of GQA: repeat each KV head G times, attend per query head, then sum the
+    # G heads of a group
+    kr = k.double().repeat_interleave(G, dim=2)  # [NL,Bt,Hq,L,D]
+    s = torch.einsum("nbhwd,nbhld->nbhwl", q.double(), kr) / math.sqrt(D)
+    c = torch.softmax(s, dim=-1).sum(3).view(NL, Bt, Hkv, G, L).sum(3)
+    np.testing.assert_allclose(out["colsum"], c.numpy(), rtol=1e-12)
+    pooled = torch.nn.functional.avg_pool1d(c[..., :L - R].reshape(-1, 1, L - R), kernel, 1,
+                                            kernel // 2).view(NL, Bt, Hkv, L - R)
+    np.testing.assert_allclose(out["scores"], pooled.numpy(), rtol=1e-12)
+    kb = k.view(torch.int16).numpy().view(np.uint16)
+    vb = v.view(torch.int16).numpy().view(np.uint16)
+    for n in range(NL):
+        for b in range(Bt):
+            for h in range(Hkv):
+                idx = out["idx"][n, b, h]
+                want = np.sort(np.argsort(-out["scores"][n, b, h], kind="stable")[:B - R])
+                assert (idx[:B - R] == want).all()
+                assert idx[B - R:].tolist() == list(range(L - R, L))
+                assert (out["k_out"][n, b, h] == kb[n, b, h][idx]).all()
+                assert (out["v_out"][n, b, h] == vb[n, b, h][idx]).all()
+
+
+def test_evict_unit_list_matches_full_run():
+    q = rand_bf16((2, 1, 4, 2, 16), 111)
+    k = rand_bf16((2, 1, 2, 40, 16), 112)
+    full = orc.evict(q, k, k, 2, 3, 10)
+    part = orc.evict(q, k, k, 2, 3, 10, units=[1, 2])
+    for u in (1, 2):
+        n, h = divmod(u, 2)
+        assert (part["idx"][n, 0, h] == full["idx"][n, 0, h]).all()
+        assert (part["scores"][n, 0, h] == full["scores"][n, 0, h]).all()
+    assert (part["idx"][0, 0, 0] == 0).all()
+
+
+def test_config1_planted_key_is_kept():
+    cfg = synth.CONFIGS[1]
+    inp = synth.make_inputs(cfg, "cpu")
+    out = orc.evict(inp["q"], inp["k"], inp["v"], cfg.keep_tail, cfg.pool_kernel, cfg.budgets[0])
+    idx = out["idx"][0, 0, 0]
+    B, R, L = cfg.budgets[0], cfg.keep_tail, cfg.prompt_len
+    assert idx.shape == (B,) and len(set(idx.tolist())) == B
+    assert idx[B - R:].tolist() == list(range(L - R, L))
+    assert int(inp["planted"]["one"][0, 0, 0]) in set(idx.tolist())
+    assert out["scores"].sum() <= cfg.rows + 1e-9
+
+
+def test_sink_and_needles_kept_when_budget_allows():
+    cfg = synth.CONFIGS[3].scaled(n_layers=1, batch=1, n_kv_heads=2, n_q_heads=8, prompt_len=2048,
+                                  window_len=8)
+    inp = synth.make_inputs(cfg, "cpu")
+    B = 8 + (cfg.n_needles + 1) * cfg.pool_kernel + 64
+    out = orc.evict(inp["q"], inp["k"], inp["v"], cfg.keep_tail, cfg.pool_kernel, B)
+    for h in range(cfg.n_kv_heads):
+        kept = set(out["idx"][0, 0, h].tolist())
+        assert 0 in kept
+        assert set(inp["planted"]["needles"][0, 0, h].tolist()) <= kept
