@@ -52,6 +52,12 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#if defined(__GNUC__)
+#define LAQ_API __attribute__((visibility("default")))
+#else
+#define LAQ_API
+#endif
+
 #ifdef __cplusplus
 extern "C" {
 #endif
@@ -93,11 +99,11 @@ typedef struct {
 } laq_params;
 
 /* Fills the stride fields of `p` for densely packed tensors in the index order shown above. */
-void laq_params_dense_strides(laq_params* p);
+LAQ_API void laq_params_dense_strides(laq_params* p);
 
 /* Bytes of caller-provided device scratch that laq_score / laq_evict need for `p`
  * (0 if `p` is invalid). laq_select and laq_compact need none. */
-size_t laq_workspace_bytes(const laq_params* p);
+LAQ_API size_t laq_workspace_bytes(const laq_params* p);
 
 /*
  * Steps 1-4 (Eq. 4's sum over the window, Section 4.3): pooled importance of every scored
@@ -108,7 +114,7 @@ size_t laq_workspace_bytes(const laq_params* p);
  *   ws      device scratch, ws_bytes >= laq_workspace_bytes(p)
  * Errors: LAQ_ERR_INVALID_ARG, LAQ_ERR_UNSUPPORTED, LAQ_ERR_WORKSPACE, LAQ_ERR_CUDA.
  */
-laq_status laq_score(const laq_params* p, const void* q, const void* k, float* scores,
+LAQ_API laq_status laq_score(const laq_params* p, const void* q, const void* k, float* scores,
                      void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
@@ -119,7 +125,7 @@ laq_status laq_score(const laq_params* p, const void* q, const void* k, float* s
  *           [0, L-R), last R entries are L-R .. L-1
  * Only n_layers, batch, n_kv_heads, prompt_len, keep_tail and budget of `p` are read.
  */
-laq_status laq_select(const laq_params* p, const float* scores, int32_t* idx, void* cuda_stream);
+LAQ_API laq_status laq_select(const laq_params* p, const float* scores, int32_t* idx, void* cuda_stream);
 
 /*
  * Step 6 ("cache re-eviction based on the given budget", Section 4.3): gathers the kept rows.
@@ -128,7 +134,7 @@ laq_status laq_select(const laq_params* p, const float* scores, int32_t* idx, vo
  *   k_out, v_out  device, bf16, [NL][Bt][Hkv][B][D] with the o_stride_* strides; either may be
  *                 NULL to skip that tensor. Must not overlap k / v.
  */
-laq_status laq_compact(const laq_params* p, const void* k, const void* v, const int32_t* idx,
+LAQ_API laq_status laq_compact(const laq_params* p, const void* k, const void* v, const int32_t* idx,
                        void* k_out, void* v_out, void* cuda_stream);
 
 /*
@@ -137,7 +143,7 @@ laq_status laq_compact(const laq_params* p, const void* k, const void* v, const 
  *   scores  optional (NULL allowed) device fp32 [NL][Bt][Hkv][L-R]: receives the pooled scores
  * Other arguments as in laq_score / laq_compact.
  */
-laq_status laq_evict(const laq_params* p, const void* q, const void* k, const void* v,
+LAQ_API laq_status laq_evict(const laq_params* p, const void* q, const void* k, const void* v,
                      void* k_out, void* v_out, int32_t* idx, float* scores, void* ws,
                      size_t ws_bytes, void* cuda_stream);
 
@@ -146,14 +152,14 @@ laq_status laq_evict(const laq_params* p, const void* q, const void* k, const vo
  * `ws` recorded on the device: LAQ_OK, LAQ_ERR_TIMEOUT (a bounded wait ran out; outputs are
  * not valid) or LAQ_ERR_CUDA (the synchronise or the read-back failed).
  */
-laq_status laq_last_device_status(const laq_params* p, const void* ws, size_t ws_bytes,
+LAQ_API laq_status laq_last_device_status(const laq_params* p, const void* ws, size_t ws_bytes,
                                   void* cuda_stream);
 
 /* Kernel launches the most recent call on this host thread enqueued (for accounting). */
-int laq_last_launch_count(void);
+LAQ_API int laq_last_launch_count(void);
 
-const char* laq_status_string(laq_status s);
-int laq_version(void);
+LAQ_API const char* laq_status_string(laq_status s);
+LAQ_API int laq_version(void);
 
 #ifdef __cplusplus
 }

@@ -1,0 +1,207 @@
+"""Thin ctypes binding of the C-ABI library ``liblaq`` (see ``include/laq.h``).
+
+Argument marshalling only: every step of the eviction path (Section 4.3, Eq. 4) runs in the
+library's CUDA kernels. PyTorch supplies device memory and the current stream. There is no CPU
+fallback: if ``liblaq.so`` has not been built, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblaq.so")
+
+LAQ_OK = 0
+LAQ_ERR_INVALID_ARG = 1
+LAQ_ERR_UNSUPPORTED = 2
+LAQ_ERR_WORKSPACE = 3
+LAQ_ERR_CUDA = 4
+LAQ_ERR_TIMEOUT = 5
+LAQ_ERR_INTERNAL = 6
+
+EXPORTS = (
+    "laq_params_dense_strides", "laq_workspace_bytes", "laq_score", "laq_select", "laq_compact",
+    "laq_evict", "laq_last_device_status", "laq_last_launch_count", "laq_status_string",
+    "laq_version",
+)
+
+
+class LaqParams(ctypes.Structure):
+    """Mirror of ``laq_params`` (field order and types as in laq.h)."""
+
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "prompt_len", "window_len",
+        "keep_tail", "pool_kernel", "pool_mode", "budget")] + [("softmax_scale", ctypes.c_float)] + [
+        (f"{t}_stride_{d}", ctypes.c_int64) for t in ("q", "k", "v", "o")
+        for d in ("layer", "batch", "head", "pos")]
+
+
+class LaqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (laq_status {status})")
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2505_20334_b200.build` "
+            "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, sz, pp = ctypes.c_void_p, ctypes.c_size_t, ctypes.POINTER(LaqParams)
+    lib.laq_params_dense_strides.argtypes = [pp]
+    lib.laq_params_dense_strides.restype = None
+    lib.laq_workspace_bytes.argtypes = [pp]
+    lib.laq_workspace_bytes.restype = sz
+    lib.laq_score.argtypes = [pp, vp, vp, vp, vp, sz, vp]
+    lib.laq_score.restype = ctypes.c_int
+    lib.laq_select.argtypes = [pp, vp, vp, vp]
+    lib.laq_select.restype = ctypes.c_int
+    lib.laq_compact.argtypes = [pp, vp, vp, vp, vp, vp, vp]
+    lib.laq_compact.restype = ctypes.c_int
+    lib.laq_evict.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.laq_evict.restype = ctypes.c_int
+    lib.laq_last_device_status.argtypes = [pp, vp, sz, vp]
+    lib.laq_last_device_status.restype = ctypes.c_int
+    lib.laq_last_launch_count.argtypes = []
+    lib.laq_last_launch_count.restype = ctypes.c_int
+    lib.laq_status_string.argtypes = [ctypes.c_int]
+    lib.laq_status_string.restype = ctypes.c_char_p
+    lib.laq_version.argtypes = []
+    lib.laq_version.restype = ctypes.c_int
+    return lib
+
+
+lib = _load()
+
+
+def status_string(status: int) -> str:
+    return lib.laq_status_string(int(status)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def make_params(n_layers, batch, n_q_heads, n_kv_heads, head_dim, prompt_len, window_len,
+                keep_tail, pool_kernel, budget, softmax_scale=0.0, q=None, k=None, v=None,
+                out=None) -> LaqParams:
+    """Fills ``laq_params``; strides are dense unless 5-D tensors are given to take them from."""
+    p = LaqParams()
+    p.n_layers, p.batch, p.n_q_heads, p.n_kv_heads = n_layers, batch, n_q_heads, n_kv_heads
+    p.head_dim, p.prompt_len, p.window_len, p.keep_tail = head_dim, prompt_len, window_len, keep_tail
+    p.pool_kernel, p.pool_mode, p.budget, p.softmax_scale = pool_kernel, 0, budget, softmax_scale
+    lib.laq_params_dense_strides(ctypes.byref(p))
+    for name, t in (("q", q), ("k", k), ("v", v), ("o", out)):
+        if t is not None:
+            if t.dim() != 5 or t.stride(4) != 1:
+                raise ValueError(f"{name}: expected a 5-D tensor with unit innermost stride")
+            for i, d in enumerate(("layer", "batch", "head", "pos")):
+                setattr(p, f"{name}_stride_{d}", t.stride(i))
+    return p
+
+
+def params_for(q: torch.Tensor, k: torch.Tensor, keep_tail: int, pool_kernel: int, budget: int,
+               v: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
+               softmax_scale: float = 0.0) -> LaqParams:
+    """``laq_params`` for q [NL,Bt,Hq,W,D] and k [NL,Bt,Hkv,L,D] (strides taken from the tensors)."""
+    NL, Bt, Hq, W, D = q.shape
+    Hkv, L = k.shape[2], k.shape[3]
+    return make_params(NL, Bt, Hq, Hkv, D, L, W, keep_tail, pool_kernel, budget, softmax_scale,
+                       q=q, k=k, v=v, out=out)
+
+
+def laq_workspace_bytes(p: LaqParams) -> int:
+    return int(lib.laq_workspace_bytes(ctypes.byref(p)))
+
+
+def alloc_workspace(p: LaqParams, device) -> torch.Tensor:
+    n = laq_workspace_bytes(p)
+    if n == 0:
+        raise LaqError(LAQ_ERR_INVALID_ARG, "laq_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def _ws_args(ws: Optional[torch.Tensor]):
+    return _ptr(ws), (0 if ws is None else ws.numel() * ws.element_size())
+
+
+def laq_score(p: LaqParams, q, k, scores, ws, stream=None, check=True) -> int:
+    wp, wn = _ws_args(ws)
+    st = lib.laq_score(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(scores), wp, wn, _stream(stream))
+    if check and st != LAQ_OK:
+        raise LaqError(st, "laq_score")
+    return st
+
+
+def laq_select(p: LaqParams, scores, idx, stream=None, check=True) -> int:
+    st = lib.laq_select(ctypes.byref(p), _ptr(scores), _ptr(idx), _stream(stream))
+    if check and st != LAQ_OK:
+        raise LaqError(st, "laq_select")
+    return st
+
+
+def laq_compact(p: LaqParams, k, v, idx, k_out, v_out, stream=None, check=True) -> int:
+    st = lib.laq_compact(ctypes.byref(p), _ptr(k), _ptr(v), _ptr(idx), _ptr(k_out), _ptr(v_out),
+                         _stream(stream))
+    if check and st != LAQ_OK:
+        raise LaqError(st, "laq_compact")
+    return st
+
+
+def laq_evict(p: LaqParams, q, k, v, k_out, v_out, idx, scores, ws, stream=None, check=True) -> int:
+    wp, wn = _ws_args(ws)
+    st = lib.laq_evict(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(k_out), _ptr(v_out),
+                       _ptr(idx), _ptr(scores), wp, wn, _stream(stream))
+    if check and st != LAQ_OK:
+        raise LaqError(st, "laq_evict")
+    return st
+
+
+def laq_last_device_status(p: LaqParams, ws, stream=None) -> int:
+    wp, wn = _ws_args(ws)
+    return int(lib.laq_last_device_status(ctypes.byref(p), wp, wn, _stream(stream)))
+
+
+def laq_last_launch_count() -> int:
+    return int(lib.laq_last_launch_count())
+
+
+def laq_version() -> int:
+    return int(lib.laq_version())
+
+
+def evict(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, budget: int, pool_kernel: int = 7,
+          keep_tail: Optional[int] = None, want_scores: bool = False, ws=None, stream=None):
+    """Convenience call: allocates the outputs with torch and runs ``laq_evict``.
+
+    q [NL,Bt,Hq,W,D], k and v [NL,Bt,Hkv,L,D], bf16 CUDA tensors. Returns a dict with 'k_out',
+    'v_out' [NL,Bt,Hkv,B,D], 'idx' [NL,Bt,Hkv,B] int32 and, if asked, 'scores' [NL,Bt,Hkv,L-R].
+    """
+    if not (q.is_cuda and k.is_cuda and v.is_cuda):
+        raise ValueError("evict: q, k and v must be CUDA tensors (there is no CPU path)")
+    NL, Bt, Hq, W, D = q.shape
+    Hkv, L = k.shape[2], k.shape[3]
+    R = W if keep_tail is None else keep_tail
+    k_out = torch.empty((NL, Bt, Hkv, budget, D), dtype=k.dtype, device=k.device)
+    v_out = torch.empty_like(k_out)
+    idx = torch.empty((NL, Bt, Hkv, budget), dtype=torch.int32, device=k.device)
+    scores = torch.empty((NL, Bt, Hkv, L - R), dtype=torch.float32, device=k.device) if want_scores else None
+    p = params_for(q, k, R, pool_kernel, budget, v=v, out=k_out)
+    if ws is None:
+        ws = alloc_workspace(p, k.device)
+    laq_evict(p, q, k, v, k_out, v_out, idx, scores, ws, stream)
+    out = {"k_out": k_out, "v_out": v_out, "idx": idx, "ws": ws, "params": p}
+    if want_scores:
+        out["scores"] = scores
+    return out

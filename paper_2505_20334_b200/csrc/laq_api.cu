@@ -1,0 +1,292 @@
+// C-ABI entry points of liblaq: host-side validation, workspace planning and stream-ordered
+// launches. Every step of the path runs in the kernels of the other translation units.
+#include <math.h>
+#include <string.h>
+
+#include "laq_internal.cuh"
+
+namespace laq {
+
+static bool mult8(int64_t x) { return x > 0 && (x % 8) == 0; }
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+laq_status derive_dims(const laq_params* p, Dims* d) {
+  if (!p) return LAQ_ERR_INVALID_ARG;
+  if (p->n_layers < 1 || p->batch < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1 ||
+      p->head_dim < 1 || p->prompt_len < 1 || p->window_len < 1)
+    return LAQ_ERR_INVALID_ARG;
+  if (p->n_q_heads % p->n_kv_heads != 0) return LAQ_ERR_INVALID_ARG;
+  if (p->keep_tail < 0 || p->keep_tail >= p->budget || p->budget >= p->prompt_len)
+    return LAQ_ERR_INVALID_ARG;
+  if (p->pool_kernel < 1 || (p->pool_kernel % 2) == 0) return LAQ_ERR_INVALID_ARG;
+  if (!(p->softmax_scale >= 0.0f) || isinf(p->softmax_scale)) return LAQ_ERR_INVALID_ARG;
+  if (p->pool_mode != LAQ_POOL_AVG) return LAQ_ERR_UNSUPPORTED;
+  if ((p->head_dim % 8) != 0 || p->head_dim > 256) return LAQ_ERR_UNSUPPORTED;
+  const int64_t M = (int64_t)(p->n_q_heads / p->n_kv_heads) * p->window_len;
+  if (M > 256) return LAQ_ERR_UNSUPPORTED;
+  d->NL = p->n_layers;
+  d->Bt = p->batch;
+  d->Hq = p->n_q_heads;
+  d->Hkv = p->n_kv_heads;
+  d->G = p->n_q_heads / p->n_kv_heads;
+  d->D = p->head_dim;
+  d->L = p->prompt_len;
+  d->W = p->window_len;
+  d->R = p->keep_tail;
+  d->kpool = p->pool_kernel;
+  d->B = p->budget;
+  d->M = (int)M;
+  d->Ls = d->L - d->R;
+  d->Kb = d->B - d->R;
+  d->U = (int64_t)d->NL * d->Bt * d->Hkv;
+  d->scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / sqrtf((float)d->D);
+  return LAQ_OK;
+}
+
+static laq_status check_strides_qk(const laq_params* p) {
+  if (!mult8(p->q_stride_layer) || !mult8(p->q_stride_batch) || !mult8(p->q_stride_head) ||
+      !mult8(p->q_stride_pos) || !mult8(p->k_stride_layer) || !mult8(p->k_stride_batch) ||
+      !mult8(p->k_stride_head) || !mult8(p->k_stride_pos))
+    return LAQ_ERR_INVALID_ARG;
+  if (p->q_stride_pos < p->head_dim || p->k_stride_pos < p->head_dim) return LAQ_ERR_INVALID_ARG;
+  return LAQ_OK;
+}
+
+static laq_status check_strides_vo(const laq_params* p, bool need_v) {
+  if (need_v && (!mult8(p->v_stride_layer) || !mult8(p->v_stride_batch) ||
+                 !mult8(p->v_stride_head) || !mult8(p->v_stride_pos) ||
+                 p->v_stride_pos < p->head_dim))
+    return LAQ_ERR_INVALID_ARG;
+  if (!mult8(p->o_stride_layer) || !mult8(p->o_stride_batch) || !mult8(p->o_stride_head) ||
+      !mult8(p->o_stride_pos) || p->o_stride_pos < p->head_dim)
+    return LAQ_ERR_INVALID_ARG;
+  if (!mult8(p->k_stride_layer) || !mult8(p->k_stride_batch) || !mult8(p->k_stride_head) ||
+      !mult8(p->k_stride_pos) || p->k_stride_pos < p->head_dim)
+    return LAQ_ERR_INVALID_ARG;
+  return LAQ_OK;
+}
+
+int choose_tiles_per_task(const Dims& d) {
+  const int n_tiles = (d.L + TILE_KEYS - 1) / TILE_KEYS;
+  int t = (n_tiles + 63) / 64;
+  if (t < 4) t = 4;
+  if (t > n_tiles) t = n_tiles;
+  return t;
+}
+
+void plan_workspace(const Dims& d, int tiles_per_task, Workspace* w) {
+  const int n_tiles = (d.L + TILE_KEYS - 1) / TILE_KEYS;
+  const int n_tasks = (n_tiles + tiles_per_task - 1) / tiles_per_task;
+  w->n_part = 2 * n_tasks;
+  w->M_pad = (d.M + 31) / 32 * 32;
+  w->L_pad = n_tiles * TILE_KEYS;
+  size_t off = 0;
+  w->off_hdr = off;
+  off = align_up(off + HDR_WORDS * sizeof(int32_t), 256);
+  w->off_cnt = off;
+  off = align_up(off + (size_t)d.U * sizeof(int32_t), 256);
+  w->off_rdy = off;
+  off = align_up(off + (size_t)d.U * sizeof(int32_t), 256);
+  w->off_part = off;
+  off = align_up(off + (size_t)d.U * w->n_part * w->M_pad * sizeof(float2), 256);
+  w->off_rowoff = off;
+  off = align_up(off + (size_t)d.U * w->M_pad * sizeof(float), 256);
+  w->off_colsum = off;
+  off = align_up(off + (size_t)d.U * w->L_pad * sizeof(float), 256);
+  w->off_pooled = off;
+  off = align_up(off + (size_t)d.U * d.Ls * sizeof(float), 256);
+  w->off_idx = off;
+  off = align_up(off + (size_t)d.U * d.B * sizeof(int32_t), 256);
+  w->total = off;
+}
+
+static bool use_tensor_core_path(const Dims& d) { return d.D == 128 && d.M <= 256; }
+
+static thread_local int g_last_launches = 0;
+
+// Steps 1-3 into the workspace's colsum array.
+static laq_status run_scoring(const laq_params* p, const Dims& d, const Workspace& w,
+                              const void* q, const void* k, char* ws, cudaStream_t stream,
+                              int* launches) {
+  // header, unit counters and ready flags are contiguous: one clear
+  if (cudaMemsetAsync(ws + w.off_hdr, 0, w.off_part - w.off_hdr, stream) != cudaSuccess)
+    return LAQ_ERR_CUDA;
+  if (use_tensor_core_path(d)) return score_tc_launch(*p, d, w, q, k, ws, stream, launches);
+  return score_simt_launch(*p, d, w, q, k, ws, stream, launches);
+}
+
+static laq_status check_ws(const Workspace& w, const void* ws, size_t ws_bytes) {
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0 || ws_bytes < w.total)
+    return LAQ_ERR_WORKSPACE;
+  return LAQ_OK;
+}
+
+}  // namespace laq
+
+using namespace laq;
+
+extern "C" {
+
+void laq_params_dense_strides(laq_params* p) {
+  if (!p) return;
+  const int64_t D = p->head_dim;
+  p->q_stride_pos = D;
+  p->q_stride_head = (int64_t)p->window_len * D;
+  p->q_stride_batch = (int64_t)p->n_q_heads * p->q_stride_head;
+  p->q_stride_layer = (int64_t)p->batch * p->q_stride_batch;
+  p->k_stride_pos = D;
+  p->k_stride_head = (int64_t)p->prompt_len * D;
+  p->k_stride_batch = (int64_t)p->n_kv_heads * p->k_stride_head;
+  p->k_stride_layer = (int64_t)p->batch * p->k_stride_batch;
+  p->v_stride_pos = p->k_stride_pos;
+  p->v_stride_head = p->k_stride_head;
+  p->v_stride_batch = p->k_stride_batch;
+  p->v_stride_layer = p->k_stride_layer;
+  p->o_stride_pos = D;
+  p->o_stride_head = (int64_t)p->budget * D;
+  p->o_stride_batch = (int64_t)p->n_kv_heads * p->o_stride_head;
+  p->o_stride_layer = (int64_t)p->batch * p->o_stride_batch;
+}
+
+size_t laq_workspace_bytes(const laq_params* p) {
+  Dims d;
+  if (derive_dims(p, &d) != LAQ_OK) return 0;
+  Workspace w;
+  plan_workspace(d, choose_tiles_per_task(d), &w);
+  return w.total;
+}
+
+laq_status laq_score(const laq_params* p, const void* q, const void* k, float* scores, void* ws,
+                     size_t ws_bytes, void* cuda_stream) {
+  g_last_launches = 0;
+  Dims d;
+  laq_status st = derive_dims(p, &d);
+  if (st != LAQ_OK) return st;
+  if (!q || !k || !scores || !aligned16(q) || !aligned16(k) ||
+      (reinterpret_cast<uintptr_t>(scores) & 3u))
+    return LAQ_ERR_INVALID_ARG;
+  if ((st = check_strides_qk(p)) != LAQ_OK) return st;
+  Workspace w;
+  plan_workspace(d, choose_tiles_per_task(d), &w);
+  if ((st = check_ws(w, ws, ws_bytes)) != LAQ_OK) return st;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  char* wsb = (char*)ws;
+  int launches = 0;
+  st = run_scoring(p, d, w, q, k, wsb, stream, &launches);
+  if (st == LAQ_OK)
+    st = pool_launch(d, (const float*)(wsb + w.off_colsum), w.L_pad, scores, stream, &launches);
+  g_last_launches = launches;
+  return st;
+}
+
+laq_status laq_select(const laq_params* p, const float* scores, int32_t* idx,
+                      void* cuda_stream) {
+  g_last_launches = 0;
+  if (!p) return LAQ_ERR_INVALID_ARG;
+  if (p->n_layers < 1 || p->batch < 1 || p->n_kv_heads < 1 || p->prompt_len < 1 ||
+      p->keep_tail < 0 || p->keep_tail >= p->budget || p->budget >= p->prompt_len)
+    return LAQ_ERR_INVALID_ARG;
+  if (!scores || !idx || (reinterpret_cast<uintptr_t>(scores) & 3u) ||
+      (reinterpret_cast<uintptr_t>(idx) & 3u))
+    return LAQ_ERR_INVALID_ARG;
+  Dims d;
+  memset(&d, 0, sizeof d);
+  d.NL = p->n_layers;
+  d.Bt = p->batch;
+  d.Hkv = p->n_kv_heads;
+  d.L = p->prompt_len;
+  d.R = p->keep_tail;
+  d.B = p->budget;
+  d.Ls = d.L - d.R;
+  d.Kb = d.B - d.R;
+  d.U = (int64_t)d.NL * d.Bt * d.Hkv;
+  int launches = 0;
+  laq_status st = select_launch(d, scores, idx, (cudaStream_t)cuda_stream, &launches);
+  g_last_launches = launches;
+  return st;
+}
+
+laq_status laq_compact(const laq_params* p, const void* k, const void* v, const int32_t* idx,
+                       void* k_out, void* v_out, void* cuda_stream) {
+  g_last_launches = 0;
+  Dims d;
+  laq_status st = derive_dims(p, &d);
+  if (st != LAQ_OK) return st;
+  if (!idx || (reinterpret_cast<uintptr_t>(idx) & 3u)) return LAQ_ERR_INVALID_ARG;
+  if ((k_out && !k) || (v_out && !v)) return LAQ_ERR_INVALID_ARG;
+  if (!aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out))
+    return LAQ_ERR_INVALID_ARG;
+  if ((st = check_strides_vo(p, v_out != nullptr)) != LAQ_OK) return st;
+  int launches = 0;
+  st = compact_launch(*p, d, k, v, idx, k_out, v_out, (cudaStream_t)cuda_stream, &launches);
+  g_last_launches = launches;
+  return st;
+}
+
+laq_status laq_evict(const laq_params* p, const void* q, const void* k, const void* v,
+                     void* k_out, void* v_out, int32_t* idx, float* scores, void* ws,
+                     size_t ws_bytes, void* cuda_stream) {
+  g_last_launches = 0;
+  Dims d;
+  laq_status st = derive_dims(p, &d);
+  if (st != LAQ_OK) return st;
+  if (!q || !k || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) ||
+      !aligned16(v_out))
+    return LAQ_ERR_INVALID_ARG;
+  if (v_out && !v) return LAQ_ERR_INVALID_ARG;
+  if (!k_out && !v_out && !idx && !scores) return LAQ_ERR_INVALID_ARG;
+  if ((scores && (reinterpret_cast<uintptr_t>(scores) & 3u)) ||
+      (idx && (reinterpret_cast<uintptr_t>(idx) & 3u)))
+    return LAQ_ERR_INVALID_ARG;
+  if ((st = check_strides_qk(p)) != LAQ_OK) return st;
+  if ((k_out || v_out) && (st = check_strides_vo(p, v_out != nullptr)) != LAQ_OK) return st;
+  Workspace w;
+  plan_workspace(d, choose_tiles_per_task(d), &w);
+  if ((st = check_ws(w, ws, ws_bytes)) != LAQ_OK) return st;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  char* wsb = (char*)ws;
+  int launches = 0;
+  st = run_scoring(p, d, w, q, k, wsb, stream, &launches);
+  float* pooled = scores ? scores : (float*)(wsb + w.off_pooled);
+  if (st == LAQ_OK)
+    st = pool_launch(d, (const float*)(wsb + w.off_colsum), w.L_pad, pooled, stream, &launches);
+  int32_t* idx_dev = idx ? idx : (int32_t*)(wsb + w.off_idx);
+  if (st == LAQ_OK && (idx || k_out || v_out))
+    st = select_launch(d, pooled, idx_dev, stream, &launches);
+  if (st == LAQ_OK && (k_out || v_out))
+    st = compact_launch(*p, d, k, v, idx_dev, k_out, v_out, stream, &launches);
+  g_last_launches = launches;
+  return st;
+}
+
+laq_status laq_last_device_status(const laq_params* p, const void* ws, size_t ws_bytes,
+                                  void* cuda_stream) {
+  Dims d;
+  laq_status st = derive_dims(p, &d);
+  if (st != LAQ_OK) return st;
+  if (!ws || ws_bytes < HDR_WORDS * sizeof(int32_t)) return LAQ_ERR_WORKSPACE;
+  if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return LAQ_ERR_CUDA;
+  int32_t hdr[HDR_WORDS];
+  if (cudaMemcpy(hdr, ws, sizeof hdr, cudaMemcpyDeviceToHost) != cudaSuccess) return LAQ_ERR_CUDA;
+  if (hdr[HDR_STATUS] == 0) return LAQ_OK;
+  return hdr[HDR_STATUS] == LAQ_ERR_TIMEOUT ? LAQ_ERR_TIMEOUT : LAQ_ERR_INTERNAL;
+}
+
+int laq_last_launch_count(void) { return g_last_launches; }
+
+const char* laq_status_string(laq_status s) {
+  switch (s) {
+    case LAQ_OK: return "ok";
+    case LAQ_ERR_INVALID_ARG: return "invalid argument";
+    case LAQ_ERR_UNSUPPORTED: return "unsupported problem shape";
+    case LAQ_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case LAQ_ERR_CUDA: return "CUDA call failed";
+    case LAQ_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    case LAQ_ERR_INTERNAL: return "internal error";
+  }
+  return "unknown status";
+}
+
+int laq_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,67 @@
+// Internal declarations shared by the translation units of liblaq (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "laq.h"
+
+namespace laq {
+
+// Problem sizes derived from laq_params (notation of laq.h).
+struct Dims {
+  int NL, Bt, Hq, Hkv, G, D, L, W, R, kpool, B;
+  int M;        // G*W softmax rows per unit
+  int Ls, Kb;   // scored positions, selected slots
+  int64_t U;    // units
+  float scale;  // softmax scale
+};
+
+// Workspace layout (all offsets in bytes from the 256-byte aligned base).
+//   header   : int32 words (see HDR_*), zeroed at the start of every scoring call
+//   unit_cnt : int32 [U]   partial row statistics delivered so far, zeroed per call
+//   unit_rdy : int32 [U]   1 once row_off of the unit is final, zeroed per call
+//   part     : float2 [U][n_part][M_pad]  partial (max, sum) in the log2 domain
+//   row_off  : float [U][M_pad]  b_r = log2e*scale*m_r + log2(l_r)
+//   colsum   : float [U][L_pad]  c_j (step 3)
+//   pooled   : float [U][Ls]     p_j (step 4) when the caller gave no scores buffer
+//   idx      : int32 [U][B]      kept positions when the caller gave no idx buffer
+struct Workspace {
+  size_t off_hdr, off_cnt, off_rdy, off_part, off_rowoff, off_colsum, off_pooled, off_idx, total;
+  int n_part;  // partial-statistics slots per unit
+  int M_pad;   // rows padded to a multiple of 32
+  int L_pad;   // L padded to a multiple of 128
+};
+
+enum { HDR_STATUS = 0, HDR_TICKET = 1, HDR_WHERE = 2, HDR_WORDS = 64 };
+
+// Keys per scoring task (a task = one sweep over KEYS_PER_TASK consecutive keys of one unit).
+constexpr int TILE_KEYS = 128;
+
+laq_status derive_dims(const laq_params* p, Dims* d);
+void plan_workspace(const Dims& d, int tiles_per_task, Workspace* w);
+int choose_tiles_per_task(const Dims& d);
+
+// Scoring back ends: both fill colsum (fp32 [U][L_pad]) on `stream`.
+// Tensor-core path (tcgen05 + TMA), head_dim 128, M <= 256.
+laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& w, const void* q,
+                           const void* k, char* ws, cudaStream_t stream, int* launches);
+// CUDA-core path for every other shape.
+laq_status score_simt_launch(const laq_params& p, const Dims& d, const Workspace& w,
+                             const void* q, const void* k, char* ws, cudaStream_t stream,
+                             int* launches);
+
+// Pool (step 4) from colsum into `pooled`.
+laq_status pool_launch(const Dims& d, const float* colsum, int L_pad, float* pooled,
+                       cudaStream_t stream, int* launches);
+// Top-k (step 5) from pooled scores.
+laq_status select_launch(const Dims& d, const float* pooled, int32_t* idx, cudaStream_t stream,
+                         int* launches);
+// Gather (step 6).
+laq_status compact_launch(const laq_params& p, const Dims& d, const void* k, const void* v,
+                          const int32_t* idx, void* k_out, void* v_out, cudaStream_t stream,
+                          int* launches);
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace laq

@@ -1,0 +1,167 @@
+// Step 4 (average pooling of the column sums) and step 5 (Eq. 4's ArgSort(...)[:B]: per-unit
+// top-k by radix select on the fp32 bit patterns, ties to the lower position, ascending output
+// followed by the retained tail).
+#include "laq_internal.cuh"
+
+namespace laq {
+namespace {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSelWarps = kSelThreads / 32;
+
+// p_j = (1/k) * sum_{|t| <= k/2, 0 <= j+t < Ls} c_{j+t}: zero padding, divisor always k.
+__global__ void pool_kernel(const float* __restrict__ colsum, int L_pad, float* __restrict__ pooled,
+                            int Ls, int kpool, float inv_k) {
+  const int64_t u = blockIdx.y;
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= Ls) return;
+  const float* c = colsum + u * L_pad;
+  const int h = kpool / 2;
+  float acc = 0.f;
+  for (int t = -h; t <= h; ++t) {
+    const int jj = j + t;
+    if (jj >= 0 && jj < Ls) acc += c[jj];
+  }
+  pooled[u * Ls + j] = acc * inv_k;
+}
+
+// Order-preserving map from fp32 bits to uint32 (larger float <=> larger key).
+__device__ __forceinline__ uint32_t order_key(float f) {
+  const uint32_t b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// One block per unit. Four 8-bit radix passes find the key of the Kb-th largest score and how
+// many positions holding exactly that key are still needed; an ordered two-step compaction then
+// writes the kept positions in ascending order.
+__global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __restrict__ pooled,
+                                                             int32_t* __restrict__ idx, int Ls,
+                                                             int Kb, int R, int B) {
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t s_prefix, s_need;
+  __shared__ uint32_t s_gt[kSelWarps], s_eq[kSelWarps];
+  const int64_t u = blockIdx.x;
+  const float* p = pooled + u * (int64_t)Ls;
+  int32_t* out = idx + u * (int64_t)B;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  if (tid == 0) {
+    s_prefix = 0;
+    s_need = (uint32_t)Kb;
+  }
+  uint32_t mask = 0;
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    if (tid < 256) hist[tid] = 0;
+    __syncthreads();
+    const uint32_t prefix = s_prefix;
+    for (int i0 = 0; i0 < Ls; i0 += kSelThreads) {
+      const int i = i0 + tid;
+      uint32_t digit = 0xffffffffu;
+      if (i < Ls) {
+        const uint32_t key = order_key(p[i]);
+        if ((key & mask) == prefix) digit = (key >> shift) & 255u;
+      }
+      // one shared-memory atomic per distinct digit in the warp
+      const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+      if (digit != 0xffffffffu && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+    }
+    __syncthreads();
+    if (warp == 0) {
+      // lane owns bins [8*lane, 8*lane+8); find the bin where the count from the top reaches need
+      uint32_t own = 0;
+#pragma unroll
+      for (int b = 0; b < 8; ++b) own += hist[lane * 8 + b];
+      uint32_t suffix = own;  // inclusive suffix sum over lanes >= lane
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_down_sync(0xffffffffu, suffix, o);
+        if (lane + o < 32) suffix += v;
+      }
+      const uint32_t above = suffix - own;
+      const uint32_t need = s_need;
+      if (above < need && need <= above + own) {
+        uint32_t acc = above;
+        for (int b = 7; b >= 0; --b) {
+          const uint32_t hcount = hist[lane * 8 + b];
+          if (acc + hcount >= need) {
+            s_prefix = prefix | ((uint32_t)(lane * 8 + b) << shift);
+            s_need = need - acc;
+            break;
+          }
+          acc += hcount;
+        }
+      }
+    }
+    mask |= 255u << shift;
+    __syncthreads();
+  }
+  const uint32_t theta = s_prefix;  // key of the Kb-th largest score
+  const uint32_t need = s_need;     // positions holding exactly theta that are kept (lowest first)
+
+  // warp w owns the contiguous positions [w*chunk, (w+1)*chunk)
+  const int chunk = ((Ls + kSelWarps - 1) / kSelWarps + 31) / 32 * 32;
+  const int beg = warp * chunk, end = min(Ls, beg + chunk);
+  uint32_t n_gt = 0, n_eq = 0;
+  for (int i0 = beg; i0 < end; i0 += 32) {
+    const int i = i0 + lane;
+    const uint32_t key = i < end ? order_key(p[i]) : 0u;
+    n_gt += __popc(__ballot_sync(0xffffffffu, i < end && key > theta));
+    n_eq += __popc(__ballot_sync(0xffffffffu, i < end && key == theta));
+  }
+  if (lane == 0) {
+    s_gt[warp] = n_gt;
+    s_eq[warp] = n_eq;
+  }
+  __syncthreads();
+  uint32_t gt_run = 0, eq_run = 0;
+  for (int w = 0; w < warp; ++w) {
+    gt_run += s_gt[w];
+    eq_run += s_eq[w];
+  }
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  for (int i0 = beg; i0 < end; i0 += 32) {
+    const int i = i0 + lane;
+    const uint32_t key = i < end ? order_key(p[i]) : 0u;
+    const bool gt = i < end && key > theta;
+    const bool eq = i < end && key == theta;
+    const uint32_t bg = __ballot_sync(0xffffffffu, gt);
+    const uint32_t be = __ballot_sync(0xffffffffu, eq);
+    const uint32_t gt_before = gt_run + __popc(bg & lt_mask);
+    const uint32_t eq_before = eq_run + __popc(be & lt_mask);
+    if (gt || (eq && eq_before < need)) out[gt_before + min(eq_before, need)] = i;
+    gt_run += __popc(bg);
+    eq_run += __popc(be);
+  }
+  for (int t = tid; t < R; t += kSelThreads) out[Kb + t] = Ls + t;
+}
+
+}  // namespace
+
+laq_status pool_launch(const Dims& d, const float* colsum, int L_pad, float* pooled,
+                       cudaStream_t stream, int* launches) {
+  if (d.U > 65535) {
+    // grid.y limit: launch in slabs of units
+    for (int64_t u0 = 0; u0 < d.U; u0 += 65535) {
+      const unsigned nu = (unsigned)((d.U - u0 < 65535) ? d.U - u0 : 65535);
+      pool_kernel<<<dim3((d.Ls + 255) / 256, nu), 256, 0, stream>>>(
+          colsum + u0 * L_pad, L_pad, pooled + u0 * d.Ls, d.Ls, d.kpool, 1.0f / (float)d.kpool);
+      *launches += 1;
+    }
+  } else {
+    pool_kernel<<<dim3((d.Ls + 255) / 256, (unsigned)d.U), 256, 0, stream>>>(
+        colsum, L_pad, pooled, d.Ls, d.kpool, 1.0f / (float)d.kpool);
+    *launches += 1;
+  }
+  return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;
+}
+
+laq_status select_launch(const Dims& d, const float* pooled, int32_t* idx, cudaStream_t stream,
+                         int* launches) {
+  if (d.U > 0x7fffffff) return LAQ_ERR_UNSUPPORTED;
+  select_kernel<<<(unsigned)d.U, kSelThreads, 0, stream>>>(pooled, idx, d.Ls, d.Kb, d.R, d.B);
+  *launches += 1;
+  return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;
+}
+
+}  // namespace laq

@@ -1,0 +1,103 @@
+"""The C-ABI library loads without a GPU, exports every symbol the header declares, and rejects
+bad arguments on the host before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2505_20334_b200 import build as laq_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def binding():
+    laq_build.build_liblaq()
+    from paper_2505_20334_b200 import binding as b
+    return b
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "laq.h")).read()
+    return sorted(set(re.findall(r"LAQ_API[^;(]*?\b(laq_\w+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported(binding):
+    names = declared_symbols()
+    assert len(names) >= 10 and "laq_evict" in names
+    raw = ctypes.CDLL(binding.LIB_PATH)
+    for n in names:
+        assert hasattr(raw, n), f"{n} declared in laq.h but not exported"
+    assert set(names) == set(binding.EXPORTS)
+
+
+def test_struct_layout_and_version(binding):
+    assert ctypes.sizeof(binding.LaqParams) == 12 * 4 + 16 * 8
+    assert binding.LaqParams.q_stride_layer.offset == 48
+    assert binding.laq_version() >= 100
+    assert binding.status_string(0) == "ok"
+    assert "argument" in binding.status_string(binding.LAQ_ERR_INVALID_ARG)
+
+
+def test_dense_strides_and_workspace(binding):
+    p = binding.make_params(2, 3, 8, 2, 128, 1000, 4, 4, 7, 64)
+    assert (p.q_stride_pos, p.q_stride_head, p.q_stride_batch, p.q_stride_layer) == (
+        128, 4 * 128, 8 * 4 * 128, 3 * 8 * 4 * 128)
+    assert (p.k_stride_pos, p.k_stride_head, p.k_stride_batch) == (128, 1000 * 128, 2 * 1000 * 128)
+    assert (p.o_stride_head, p.o_stride_layer) == (64 * 128, 3 * 2 * 64 * 128)
+    n = binding.laq_workspace_bytes(p)
+    assert n > 2 * 3 * 2 * 1000 * 4 and n % 256 == 0
+    # config 5 pool: offsets beyond 2^32 bytes must not overflow
+    big = binding.make_params(80, 1, 64, 8, 128, 65536, 32, 32, 7, 2048)
+    assert big.k_stride_layer * 80 * 2 > 2 ** 32
+    assert binding.laq_workspace_bytes(big) > 80 * 8 * 65536 * 4
+
+
+@pytest.mark.parametrize("kw", [
+    dict(n_q_heads=7),            # not a multiple of n_kv_heads
+    dict(budget=1000),            # B >= L
+    dict(budget=4),               # B <= R
+    dict(pool_kernel=4),          # even kernel
+    dict(keep_tail=-1),
+    dict(prompt_len=0),
+    dict(softmax_scale=float("nan")),
+])
+def test_invalid_params_rejected_on_host(binding, kw):
+    args = dict(n_layers=1, batch=1, n_q_heads=8, n_kv_heads=2, head_dim=128, prompt_len=1000,
+                window_len=4, keep_tail=4, pool_kernel=7, budget=64)
+    args.update(kw)
+    p = binding.make_params(**args)
+    assert binding.laq_workspace_bytes(p) == 0
+    fake = ctypes.c_void_p(4096)
+    st = binding.lib.laq_evict(ctypes.byref(p), fake, fake, fake, fake, fake, fake, None, fake,
+                               1 << 40, None)
+    assert st == binding.LAQ_ERR_INVALID_ARG
+
+
+def test_unsupported_and_pointer_checks(binding):
+    p = binding.make_params(1, 1, 8, 2, 100, 1000, 4, 4, 7, 64)   # head_dim not a multiple of 8
+    fake = ctypes.c_void_p(4096)
+    st = binding.lib.laq_evict(ctypes.byref(p), fake, fake, fake, fake, fake, fake, None, fake,
+                               1 << 40, None)
+    assert st == binding.LAQ_ERR_UNSUPPORTED
+    p = binding.make_params(1, 1, 64, 1, 128, 1000, 8, 8, 7, 64)  # G*W = 512 rows
+    assert binding.lib.laq_score(ctypes.byref(p), fake, fake, fake, fake, 1 << 40, None) == \
+        binding.LAQ_ERR_UNSUPPORTED
+    p = binding.make_params(1, 1, 8, 2, 128, 1000, 4, 4, 7, 64)
+    odd = ctypes.c_void_p(4096 + 8)
+    assert binding.lib.laq_score(ctypes.byref(p), None, fake, fake, fake, 1 << 40, None) == \
+        binding.LAQ_ERR_INVALID_ARG
+    assert binding.lib.laq_score(ctypes.byref(p), odd, fake, fake, fake, 1 << 40, None) == \
+        binding.LAQ_ERR_INVALID_ARG
+    assert binding.lib.laq_score(ctypes.byref(p), fake, fake, fake, fake, 16, None) == \
+        binding.LAQ_ERR_WORKSPACE
+    assert binding.lib.laq_score(ctypes.byref(p), fake, fake, fake, None, 0, None) == \
+        binding.LAQ_ERR_WORKSPACE
+    p.k_stride_pos = 132  # not a multiple of 8 elements
+    assert binding.lib.laq_score(ctypes.byref(p), fake, fake, fake, fake, 1 << 40, None) == \
+        binding.LAQ_ERR_INVALID_ARG
+    p = binding.make_params(1, 1, 8, 2, 128, 1000, 4, 4, 7, 64)
+    assert binding.lib.laq_select(ctypes.byref(p), None, fake, None) == binding.LAQ_ERR_INVALID_ARG
+    assert binding.lib.laq_compact(ctypes.byref(p), fake, fake, None, fake, fake, None) == \
+        binding.LAQ_ERR_INVALID_ARG

@@ -1,0 +1,257 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle on the same
+seeded inputs. Scores within 2e-3 relative; selection bit-exact on identical scores and equal to
+the oracle's set outside the tie band; compaction bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import laq_oracle as orc
+from paper_2505_20334_b200 import synth
+from parity_util import SCORE_RTOL, bits, check_index_set, score_rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def laq():
+    from paper_2505_20334_b200 import build
+    build.build_liblaq()
+    from paper_2505_20334_b200 import binding
+    return binding
+
+
+def rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed, kscale=1.0):
+    g = torch.Generator().manual_seed(seed)
+    q = torch.randn((NL, Bt, Hq, W, D), generator=g).to(torch.bfloat16)
+    k = (torch.randn((NL, Bt, Hkv, L, D), generator=g) * kscale).to(torch.bfloat16)
+    v = torch.randn((NL, Bt, Hkv, L, D), generator=g).to(torch.bfloat16)
+    return q, k, v
+
+
+def run_evict(laq, q, k, v, R, kernel, B):
+    out = laq.evict(q.cuda(), k.cuda(), v.cuda(), B, pool_kernel=kernel, keep_tail=R,
+                    want_scores=True)
+    assert laq.laq_last_device_status(out["params"], out["ws"]) == laq.LAQ_OK
+    return out
+
+
+def compare_all_units(laq, q, k, v, R, kernel, B, out=None):
+    """Full comparison of every unit of a (small) problem against the oracle."""
+    out = out or run_evict(laq, q, k, v, R, kernel, B)
+    ref = orc.evict(q, k, v, R, kernel, B)
+    NL, Bt, Hkv, L = k.shape[0], k.shape[1], k.shape[2], k.shape[3]
+    got_scores = out["scores"].cpu().numpy()
+    err = score_rel_err(got_scores, ref["scores"])
+    assert err <= SCORE_RTOL, f"score rel err {err:.3e}"
+    got_idx = out["idx"].cpu().numpy()
+    kb, vb = bits(k), bits(v)
+    ko, vo = bits(out["k_out"]), bits(out["v_out"])
+    differing = 0
+    for n in range(NL):
+        for b in range(Bt):
+            for h in range(Hkv):
+                differing += check_index_set(got_idx[n, b, h], ref["idx"][n, b, h],
+                                             ref["scores"][n, b, h], L, R, B)
+                # selection is bit-exact on the GPU's own scores (tie-break included)
+                want = orc.select(got_scores[n, b, h], L, R, B, sorted_variant=True)
+                assert (got_idx[n, b, h] == want).all()
+                # compaction is bit-exact given the indices
+                assert (ko[n, b, h] == kb[n, b, h][got_idx[n, b, h]]).all()
+                assert (vo[n, b, h] == vb[n, b, h][got_idx[n, b, h]]).all()
+    return err, differing
+
+
+SHAPES = [
+    # NL Bt Hq Hkv D    L     W  k  B     what
+    (1, 1, 4, 1, 128, 1024, 8, 7, 128),    # config-1 geometry, M = 32
+    (2, 1, 8, 2, 128, 1000, 16, 7, 100),   # M = 64, ragged last tile
+    (1, 2, 8, 2, 128, 777, 32, 7, 200),    # M = 128
+    (1, 1, 8, 1, 128, 1500, 32, 5, 64),    # M = 256
+    (1, 1, 2, 2, 128, 300, 8, 3, 40),      # G = 1, M = 8
+    (1, 1, 6, 2, 128, 640, 5, 3, 33),      # M = 15 (not a multiple of 16)
+    (1, 1, 4, 2, 128, 50, 4, 7, 20),       # L smaller than one tile
+    (1, 1, 8, 2, 64, 500, 8, 7, 90),       # head_dim 64: CUDA-core path
+    (1, 1, 4, 1, 256, 260, 8, 5, 48),      # head_dim 256: CUDA-core path
+]
+
+
+@pytest.mark.parametrize("shape", SHAPES, ids=[f"L{s[5]}-M{s[2] // s[3] * s[6]}-D{s[4]}" for s in SHAPES])
+def test_evict_matches_oracle_small(laq, shape):
+    NL, Bt, Hq, Hkv, D, L, W, kernel, B = shape
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=L + W, kscale=1.5)
+    err, _ = compare_all_units(laq, q, k, v, W, kernel, B)
+    assert err < SCORE_RTOL
+
+
+def test_score_select_compact_entry_points_agree_with_evict(laq):
+    NL, Bt, Hq, Hkv, D, L, W, kernel, B = 2, 2, 8, 2, 128, 900, 8, 7, 150
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=5)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    fused = run_evict(laq, q, k, v, W, kernel, B)
+    p = laq.params_for(qd, kd, W, kernel, B, v=vd)
+    ws = laq.alloc_workspace(p, "cuda")
+    scores = torch.empty((NL, Bt, Hkv, L - W), dtype=torch.float32, device="cuda")
+    idx = torch.empty((NL, Bt, Hkv, B), dtype=torch.int32, device="cuda")
+    k_out = torch.empty((NL, Bt, Hkv, B, D), dtype=torch.bfloat16, device="cuda")
+    v_out = torch.empty_like(k_out)
+    laq.laq_score(p, qd, kd, scores, ws)
+    laq.laq_select(p, scores, idx)
+    laq.laq_compact(p, kd, vd, idx, k_out, v_out)
+    torch.cuda.synchronize()
+    assert torch.equal(scores, fused["scores"])
+    assert torch.equal(idx, fused["idx"])
+    assert torch.equal(k_out, fused["k_out"]) and torch.equal(v_out, fused["v_out"])
+    # evict without the optional outputs
+    laq.laq_evict(p, qd, kd, vd, k_out.zero_(), v_out.zero_(), None, None, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(k_out, fused["k_out"]) and torch.equal(v_out, fused["v_out"])
+
+
+def test_select_bit_exact_on_ties_and_edges(laq):
+    rng = np.random.default_rng(3)
+    cases = []
+    for Ls, R, Kb in [(1000, 8, 1), (1000, 0, 999), (5000, 16, 700), (37, 3, 10), (70000, 32, 2016),
+                      (4096, 0, 128)]:
+        for kind in ("ties", "const", "random", "tiny"):
+            if kind == "ties":
+                s = rng.integers(0, 5, Ls).astype(np.float32) * 0.25
+            elif kind == "const":
+                s = np.full(Ls, 0.125, np.float32)
+            elif kind == "random":
+                s = rng.random(Ls).astype(np.float32)
+            else:
+                s = (rng.random(Ls) * 1e-30).astype(np.float32)
+                s[::7] = 0.0
+            cases.append((Ls, R, Kb, s))
+    for Ls, R, Kb, s in cases:
+        L, B = Ls + R, Kb + R
+        p = laq.make_params(1, 1, 1, 1, 128, L, 1, R, 1, B)
+        sd = torch.from_numpy(s).cuda()
+        idx = torch.empty(B, dtype=torch.int32, device="cuda")
+        laq.laq_select(p, sd, idx)
+        want = orc.select(s, L, R, B, sorted_variant=True)
+        assert (idx.cpu().numpy() == want).all(), (Ls, R, Kb)
+
+
+def test_compact_strided_layouts_bit_exact(laq):
+    NL, Bt, Hkv, L, D, B = 2, 2, 3, 200, 128, 37
+    g = torch.Generator().manual_seed(9)
+    # K stored [NL][Bt][L][Hkv][D] (position-major), V dense; output with padded head stride
+    k_store = torch.randn((NL, Bt, L, Hkv, D), generator=g).to(torch.bfloat16).cuda()
+    k = k_store.permute(0, 1, 3, 2, 4)
+    v = torch.randn((NL, Bt, Hkv, L, D), generator=g).to(torch.bfloat16).cuda()
+    idx = torch.stack([torch.randperm(L, generator=g)[:B].sort().values
+                       for _ in range(NL * Bt * Hkv)]).view(NL, Bt, Hkv, B).to(torch.int32).cuda()
+    out_store = torch.zeros((NL, Bt, Hkv, B + 5, D), dtype=torch.bfloat16, device="cuda")
+    k_out = out_store[:, :, :, :B]
+    v_store = torch.zeros_like(out_store)
+    v_out = v_store[:, :, :, :B]
+    p = laq.make_params(NL, Bt, Hkv, Hkv, D, L, 4, 4, 1, B, k=k, v=v, out=k_out)
+    laq.laq_compact(p, k, v, idx, k_out, v_out)
+    torch.cuda.synchronize()
+    gather = idx.long()[..., None].expand(-1, -1, -1, -1, D)
+    assert torch.equal(k_out, torch.gather(k, 3, gather))
+    assert torch.equal(v_out, torch.gather(v, 3, gather))
+    assert (out_store[:, :, :, B:] == 0).all()
+
+
+def test_strided_kv_cache_layout(laq):
+    # K/V kept position-major ([NL][Bt][L][Hkv][D]) as many serving engines store them
+    NL, Bt, Hq, Hkv, D, L, W, kernel, B = 1, 2, 8, 2, 128, 600, 8, 7, 64
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=77)
+    ks = k.permute(0, 1, 3, 2, 4).contiguous().cuda().permute(0, 1, 3, 2, 4)
+    vs = v.permute(0, 1, 3, 2, 4).contiguous().cuda().permute(0, 1, 3, 2, 4)
+    assert not ks.is_contiguous()
+    out = laq.evict(q.cuda(), ks, vs, B, pool_kernel=kernel, keep_tail=W, want_scores=True)
+    compare_all_units(laq, q, k, v, W, kernel, B, out=out)
+
+
+def test_edge_budgets_and_no_pooling(laq):
+    q, k, v = rand_inputs(1, 1, 4, 2, 128, 400, 4, seed=13)
+    compare_all_units(laq, q, k, v, 4, 1, 5)        # Kb = 1, no pooling
+    compare_all_units(laq, q, k, v, 0, 7, 399)      # R = 0, keep all but one
+    compare_all_units(laq, q, k, v, 4, 9, 399)      # Kb = Ls - 1
+    q, k, v = rand_inputs(1, 1, 2, 1, 128, 12, 2, seed=14)
+    compare_all_units(laq, q, k, v, 2, 15, 5)       # pool kernel wider than the scored range
+
+
+def test_workspace_reuse_back_to_back(laq):
+    q, k, v = rand_inputs(2, 1, 8, 2, 128, 1300, 8, seed=21)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    a = laq.evict(qd, kd, vd, 100, want_scores=True)
+    b = laq.evict(qd, kd, vd, 100, want_scores=True, ws=a["ws"])
+    c = laq.evict(qd, kd, vd, 100, want_scores=True, ws=a["ws"])
+    torch.cuda.synchronize()
+    assert torch.equal(a["scores"], b["scores"]) and torch.equal(a["idx"], c["idx"])
+    assert torch.equal(a["k_out"], c["k_out"])
+
+
+# ---------------------------------------------------------------- the paper-shaped configs
+def test_config1_full_with_planted_key(laq):
+    cfg = synth.CONFIGS[1]
+    inp = synth.make_inputs(cfg, "cpu")
+    B = cfg.budgets[0]
+    out = run_evict(laq, inp["q"], inp["k"], inp["v"], cfg.keep_tail, cfg.pool_kernel, B)
+    compare_all_units(laq, inp["q"], inp["k"], inp["v"], cfg.keep_tail, cfg.pool_kernel, B, out=out)
+    assert int(inp["planted"]["one"][0, 0, 0]) in set(out["idx"][0, 0, 0].tolist())
+
+
+def sampled_parity(laq, cfg, budgets, units, device="cuda"):
+    """Runs the full-size problem on the GPU and checks the listed units against the oracle."""
+    inp = synth.make_inputs(cfg, device)
+    q, k, v = inp["q"], inp["k"], inp["v"]
+    R, L, D = cfg.keep_tail, cfg.prompt_len, cfg.head_dim
+    NL, Bt, Hkv = cfg.n_layers, cfg.batch, cfg.n_kv_heads
+    worst = 0.0
+    ws = None
+    for B in budgets:
+        k_out = torch.empty((NL, Bt, Hkv, B, D), dtype=torch.bfloat16, device=k.device)
+        v_out = torch.empty_like(k_out)
+        idx = torch.empty((NL, Bt, Hkv, B), dtype=torch.int32, device=k.device)
+        scores = torch.empty((NL, Bt, Hkv, L - R), dtype=torch.float32, device=k.device)
+        p = laq.params_for(q, k, R, cfg.pool_kernel, B, v=v, out=k_out)
+        if ws is None or ws.numel() < laq.laq_workspace_bytes(p):
+            ws = laq.alloc_workspace(p, k.device)
+        laq.laq_evict(p, q, k, v, k_out, v_out, idx, scores, ws)
+        assert laq.laq_last_device_status(p, ws) == laq.LAQ_OK
+        for u in units:
+            h, b, n = u % Hkv, (u // Hkv) % Bt, u // (Hkv * Bt)
+            qu, ku, vu = synth.unit_slices(cfg, inp, u)
+            ref = orc.evict(qu, ku, vu, R, cfg.pool_kernel, B)
+            got_s = scores[n, b, h].cpu().numpy()
+            err = score_rel_err(got_s, ref["scores"][0, 0, 0])
+            worst = max(worst, err)
+            assert err <= SCORE_RTOL, f"unit {u} B {B}: score rel err {err:.3e}"
+            gi = idx[n, b, h].cpu().numpy()
+            check_index_set(gi, ref["idx"][0, 0, 0], ref["scores"][0, 0, 0], L, R, B)
+            assert (gi == orc.select(got_s, L, R, B, sorted_variant=True)).all()
+            assert (bits(k_out[n, b, h]) == bits(ku[0, 0, 0])[gi]).all()
+            assert (bits(v_out[n, b, h]) == bits(vu[0, 0, 0])[gi]).all()
+            if "sink" in inp["planted"]:
+                assert 0 in set(gi.tolist())
+            if "needles" in inp["planted"] and B - R >= (cfg.n_needles + 1) * cfg.pool_kernel:
+                assert set(inp["planted"]["needles"][n, b, h].tolist()) <= set(gi.tolist())
+    return worst
+
+
+def test_config2_full_size_sampled_units(laq):
+    cfg = synth.CONFIGS[2]
+    sampled_parity(laq, cfg, cfg.budgets, synth.sample_units(cfg, 4))
+
+
+def test_config3_full_size_sampled_units(laq):
+    cfg = synth.CONFIGS[3]
+    units = [0, 5, cfg.units // 2 + 3, cfg.units - 1]
+    sampled_parity(laq, cfg, (128, 2048), units)
+
+
+def test_config4_full_size_sampled_units(laq):
+    cfg = synth.CONFIGS[4]
+    units = [0, 777, cfg.units - 1]
+    sampled_parity(laq, cfg, cfg.budgets, units)
+
+
+def test_config5_full_size_one_pool(laq):
+    cfg = synth.CONFIGS[5]
+    units = [1, cfg.units - 1]  # the last unit's keys lie beyond 2^32 bytes from the base
+    sampled_parity(laq, cfg, (2048,), units)
