@@ -88,6 +88,9 @@ typedef struct {
   int32_t pool_mode;   /* laq_pool_mode */
   int32_t budget;      /* B, R < B < L */
   float softmax_scale; /* 0 selects 1/sqrt(head_dim) */
+  /* Scheduling knobs of the scoring kernel; 0 lets the library choose. */
+  int32_t tiles_per_task;  /* 128-key tiles per scoring task (a task = one sweep over a key chunk) */
+  int32_t sched_lag_units; /* how many units the column-sum sweep trails the statistics sweep */
   /* Q [NL][Bt][Hq][W][D] */
   int64_t q_stride_layer, q_stride_batch, q_stride_head, q_stride_pos;
   /* K [NL][Bt][Hkv][L][D] */
@@ -148,12 +151,39 @@ LAQ_API laq_status laq_evict(const laq_params* p, const void* q, const void* k, 
                      size_t ws_bytes, void* cuda_stream);
 
 /*
+ * The whole step for a cache that lives in HOST memory (ideally pinned): copies Q, K and V to the
+ * caller's device staging area, runs laq_evict there and copies the compressed cache back, all
+ * ordered on `cuda_stream`. Host tensors are densely packed in the index order of laq_params (the
+ * stride fields of `p` are ignored and dense strides are used on both sides).
+ *   q_host, k_host, v_host          HOST, bf16, inputs
+ *   k_out_host, v_out_host          HOST, bf16 [NL][Bt][Hkv][B][D], outputs
+ *   idx_host                        HOST, int32 [NL][Bt][Hkv][B], output (may be NULL)
+ *   staging, staging_bytes          DEVICE scratch of at least laq_host_staging_bytes(p) bytes,
+ *                                   256-byte aligned
+ *   ws, ws_bytes                    DEVICE workspace as for laq_evict
+ * Returns after enqueueing; the host outputs are valid once the stream has been synchronised.
+ */
+LAQ_API size_t laq_host_staging_bytes(const laq_params* p);
+LAQ_API laq_status laq_evict_host(const laq_params* p, const void* q_host, const void* k_host,
+                                  const void* v_host, void* k_out_host, void* v_out_host,
+                                  int32_t* idx_host, void* staging, size_t staging_bytes, void* ws,
+                                  size_t ws_bytes, void* cuda_stream);
+
+/*
  * Synchronises `cuda_stream` and reports what the last laq_score / laq_evict call that used
  * `ws` recorded on the device: LAQ_OK, LAQ_ERR_TIMEOUT (a bounded wait ran out; outputs are
  * not valid) or LAQ_ERR_CUDA (the synchronise or the read-back failed).
  */
 LAQ_API laq_status laq_last_device_status(const laq_params* p, const void* ws, size_t ws_bytes,
                                   void* cuda_stream);
+
+/*
+ * Instrumentation for benchmarks: caller-owned CUDA events (cudaEvent_t passed as void*) that
+ * later laq_score / laq_evict calls made by this host thread record on their stream immediately
+ * before and after the scoring kernel (steps 1-3). Pass NULL, NULL to stop recording. The events
+ * must outlive the calls that record them.
+ */
+LAQ_API void laq_set_stage_events(void* score_begin, void* score_end);
 
 /* Kernel launches the most recent call on this host thread enqueued (for accounting). */
 LAQ_API int laq_last_launch_count(void);

@@ -26,7 +26,7 @@ LAQ_ERR_INTERNAL = 6
 EXPORTS = (
     "laq_params_dense_strides", "laq_workspace_bytes", "laq_score", "laq_select", "laq_compact",
     "laq_evict", "laq_last_device_status", "laq_last_launch_count", "laq_status_string",
-    "laq_version",
+    "laq_version", "laq_set_stage_events", "laq_host_staging_bytes", "laq_evict_host",
 )
 
 
@@ -35,7 +35,8 @@ class LaqParams(ctypes.Structure):
 
     _fields_ = [(n, ctypes.c_int32) for n in (
         "n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "prompt_len", "window_len",
-        "keep_tail", "pool_kernel", "pool_mode", "budget")] + [("softmax_scale", ctypes.c_float)] + [
+        "keep_tail", "pool_kernel", "pool_mode", "budget")] + [("softmax_scale", ctypes.c_float),
+        ("tiles_per_task", ctypes.c_int32), ("sched_lag_units", ctypes.c_int32)] + [
         (f"{t}_stride_{d}", ctypes.c_int64) for t in ("q", "k", "v", "o")
         for d in ("layer", "batch", "head", "pos")]
 
@@ -71,6 +72,12 @@ def _load() -> ctypes.CDLL:
     lib.laq_last_launch_count.restype = ctypes.c_int
     lib.laq_status_string.argtypes = [ctypes.c_int]
     lib.laq_status_string.restype = ctypes.c_char_p
+    lib.laq_host_staging_bytes.argtypes = [pp]
+    lib.laq_host_staging_bytes.restype = sz
+    lib.laq_evict_host.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, sz, vp, sz, vp]
+    lib.laq_evict_host.restype = ctypes.c_int
+    lib.laq_set_stage_events.argtypes = [vp, vp]
+    lib.laq_set_stage_events.restype = None
     lib.laq_version.argtypes = []
     lib.laq_version.restype = ctypes.c_int
     return lib
@@ -177,6 +184,13 @@ def laq_last_launch_count() -> int:
     return int(lib.laq_last_launch_count())
 
 
+def laq_set_stage_events(begin=None, end=None) -> None:
+    """begin/end: recorded torch.cuda.Event objects (enable_timing=True) or None to clear."""
+    b = None if begin is None else ctypes.c_void_p(begin.cuda_event)
+    e = None if end is None else ctypes.c_void_p(end.cuda_event)
+    lib.laq_set_stage_events(b, e)
+
+
 def laq_version() -> int:
     return int(lib.laq_version())
 
@@ -205,3 +219,48 @@ def evict(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, budget: int, pool_k
     if want_scores:
         out["scores"] = scores
     return out
+
+
+
+def laq_host_staging_bytes(p: LaqParams) -> int:
+    return int(lib.laq_host_staging_bytes(ctypes.byref(p)))
+
+
+def laq_evict_host(p: LaqParams, q_host, k_host, v_host, k_out_host, v_out_host, idx_host, staging,
+                   ws, stream=None, check=True) -> int:
+    """Host tensors in, host tensors out (see laq.h); `staging` and `ws` are CUDA byte tensors."""
+    sp, sn = _ws_args(staging)
+    wp, wn = _ws_args(ws)
+    st = lib.laq_evict_host(ctypes.byref(p), _ptr(q_host), _ptr(k_host), _ptr(v_host),
+                            _ptr(k_out_host), _ptr(v_out_host), _ptr(idx_host), sp, sn, wp, wn,
+                            _stream(stream))
+    if check and st != LAQ_OK:
+        raise LaqError(st, "laq_evict_host")
+    return st
+
+
+class HostEvictor:
+    """Buffers for repeated ``laq_evict_host`` calls on one problem shape: device staging and
+    workspace, pinned host outputs. Only moves bytes; every step of the path runs in the kernels."""
+
+    def __init__(self, q_shape, k_shape, budget: int, pool_kernel: int = 7,
+                 keep_tail: Optional[int] = None, device="cuda"):
+        NL, Bt, Hq, W, D = q_shape
+        Hkv, L = k_shape[2], k_shape[3]
+        R = W if keep_tail is None else keep_tail
+        self.params = make_params(NL, Bt, Hq, Hkv, D, L, W, R, pool_kernel, budget)
+        self.ws = alloc_workspace(self.params, device)
+        self.staging = torch.empty(laq_host_staging_bytes(self.params), dtype=torch.uint8, device=device)
+        self.h_k_out = torch.empty((NL, Bt, Hkv, budget, D), dtype=torch.bfloat16, pin_memory=True)
+        self.h_v_out = torch.empty_like(self.h_k_out).pin_memory()
+        self.h_idx = torch.empty((NL, Bt, Hkv, budget), dtype=torch.int32, pin_memory=True)
+        self.h2d_bytes = 2 * (NL * Bt * Hq * W * D + 2 * NL * Bt * Hkv * L * D)
+        self.d2h_bytes = 2 * 2 * self.h_k_out.numel() + 4 * self.h_idx.numel()
+
+    def run(self, q_host, k_host, v_host, stream=None):
+        for t in (q_host, k_host, v_host):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError("laq_evict_host takes dense host tensors")
+        laq_evict_host(self.params, q_host, k_host, v_host, self.h_k_out, self.h_v_out, self.h_idx,
+                       self.staging, self.ws, stream)
+        return self.h_k_out, self.h_v_out, self.h_idx

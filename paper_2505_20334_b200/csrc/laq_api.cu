@@ -20,6 +20,7 @@ laq_status derive_dims(const laq_params* p, Dims* d) {
     return LAQ_ERR_INVALID_ARG;
   if (p->pool_kernel < 1 || (p->pool_kernel % 2) == 0) return LAQ_ERR_INVALID_ARG;
   if (!(p->softmax_scale >= 0.0f) || isinf(p->softmax_scale)) return LAQ_ERR_INVALID_ARG;
+  if (p->tiles_per_task < 0 || p->sched_lag_units < 0) return LAQ_ERR_INVALID_ARG;
   if (p->pool_mode != LAQ_POOL_AVG) return LAQ_ERR_UNSUPPORTED;
   if ((p->head_dim % 8) != 0 || p->head_dim > 256) return LAQ_ERR_UNSUPPORTED;
   const int64_t M = (int64_t)(p->n_q_heads / p->n_kv_heads) * p->window_len;
@@ -39,6 +40,8 @@ laq_status derive_dims(const laq_params* p, Dims* d) {
   d->Ls = d->L - d->R;
   d->Kb = d->B - d->R;
   d->U = (int64_t)d->NL * d->Bt * d->Hkv;
+  d->tiles_per_task = p->tiles_per_task;
+  d->sched_lag_units = p->sched_lag_units;
   d->scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / sqrtf((float)d->D);
   return LAQ_OK;
 }
@@ -68,8 +71,8 @@ static laq_status check_strides_vo(const laq_params* p, bool need_v) {
 
 int choose_tiles_per_task(const Dims& d) {
   const int n_tiles = (d.L + TILE_KEYS - 1) / TILE_KEYS;
-  int t = (n_tiles + 63) / 64;
-  if (t < 4) t = 4;
+  int t = d.tiles_per_task > 0 ? d.tiles_per_task : (n_tiles + 63) / 64;
+  if (d.tiles_per_task <= 0 && t < 4) t = 4;
   if (t > n_tiles) t = n_tiles;
   return t;
 }
@@ -103,6 +106,7 @@ void plan_workspace(const Dims& d, int tiles_per_task, Workspace* w) {
 static bool use_tensor_core_path(const Dims& d) { return d.D == 128 && d.M <= 256; }
 
 static thread_local int g_last_launches = 0;
+static thread_local cudaEvent_t g_ev_begin = nullptr, g_ev_end = nullptr;
 
 // Steps 1-3 into the workspace's colsum array.
 static laq_status run_scoring(const laq_params* p, const Dims& d, const Workspace& w,
@@ -111,8 +115,12 @@ static laq_status run_scoring(const laq_params* p, const Dims& d, const Workspac
   // header, unit counters and ready flags are contiguous: one clear
   if (cudaMemsetAsync(ws + w.off_hdr, 0, w.off_part - w.off_hdr, stream) != cudaSuccess)
     return LAQ_ERR_CUDA;
-  if (use_tensor_core_path(d)) return score_tc_launch(*p, d, w, q, k, ws, stream, launches);
-  return score_simt_launch(*p, d, w, q, k, ws, stream, launches);
+  if (g_ev_begin && cudaEventRecord(g_ev_begin, stream) != cudaSuccess) return LAQ_ERR_CUDA;
+  const laq_status st = use_tensor_core_path(d)
+                            ? score_tc_launch(*p, d, w, q, k, ws, stream, launches)
+                            : score_simt_launch(*p, d, w, q, k, ws, stream, launches);
+  if (g_ev_end && cudaEventRecord(g_ev_end, stream) != cudaSuccess) return LAQ_ERR_CUDA;
+  return st;
 }
 
 static laq_status check_ws(const Workspace& w, const void* ws, size_t ws_bytes) {
@@ -259,6 +267,66 @@ laq_status laq_evict(const laq_params* p, const void* q, const void* k, const vo
   return st;
 }
 
+struct HostStaging {
+  size_t off_q, off_k, off_v, off_ko, off_vo, off_idx, total;
+  size_t q_bytes, kv_bytes, out_bytes, idx_bytes;
+};
+
+static void plan_staging(const Dims& d, HostStaging* h) {
+  h->q_bytes = (size_t)d.NL * d.Bt * d.Hq * d.W * d.D * 2;
+  h->kv_bytes = (size_t)d.U * d.L * d.D * 2;
+  h->out_bytes = (size_t)d.U * d.B * d.D * 2;
+  h->idx_bytes = (size_t)d.U * d.B * sizeof(int32_t);
+  size_t off = 0;
+  h->off_q = off;   off = align_up(off + h->q_bytes, 256);
+  h->off_k = off;   off = align_up(off + h->kv_bytes, 256);
+  h->off_v = off;   off = align_up(off + h->kv_bytes, 256);
+  h->off_ko = off;  off = align_up(off + h->out_bytes, 256);
+  h->off_vo = off;  off = align_up(off + h->out_bytes, 256);
+  h->off_idx = off; off = align_up(off + h->idx_bytes, 256);
+  h->total = off;
+}
+
+size_t laq_host_staging_bytes(const laq_params* p) {
+  Dims d;
+  if (derive_dims(p, &d) != LAQ_OK) return 0;
+  HostStaging h;
+  plan_staging(d, &h);
+  return h.total;
+}
+
+laq_status laq_evict_host(const laq_params* p, const void* q_host, const void* k_host,
+                          const void* v_host, void* k_out_host, void* v_out_host,
+                          int32_t* idx_host, void* staging, size_t staging_bytes, void* ws,
+                          size_t ws_bytes, void* cuda_stream) {
+  g_last_launches = 0;
+  Dims d;
+  laq_status st = derive_dims(p, &d);
+  if (st != LAQ_OK) return st;
+  if (!q_host || !k_host || !v_host || !k_out_host || !v_out_host) return LAQ_ERR_INVALID_ARG;
+  HostStaging h;
+  plan_staging(d, &h);
+  if (!staging || (reinterpret_cast<uintptr_t>(staging) & 255u) != 0 || staging_bytes < h.total)
+    return LAQ_ERR_WORKSPACE;
+  laq_params dp = *p;
+  laq_params_dense_strides(&dp);
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  char* sb = (char*)staging;
+  if (cudaMemcpyAsync(sb + h.off_q, q_host, h.q_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaMemcpyAsync(sb + h.off_k, k_host, h.kv_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaMemcpyAsync(sb + h.off_v, v_host, h.kv_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    return LAQ_ERR_CUDA;
+  st = laq_evict(&dp, sb + h.off_q, sb + h.off_k, sb + h.off_v, sb + h.off_ko, sb + h.off_vo,
+                 (int32_t*)(sb + h.off_idx), nullptr, ws, ws_bytes, cuda_stream);
+  if (st != LAQ_OK) return st;
+  if (cudaMemcpyAsync(k_out_host, sb + h.off_ko, h.out_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaMemcpyAsync(v_out_host, sb + h.off_vo, h.out_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      (idx_host && cudaMemcpyAsync(idx_host, sb + h.off_idx, h.idx_bytes, cudaMemcpyDeviceToHost,
+                                   stream) != cudaSuccess))
+    return LAQ_ERR_CUDA;
+  return LAQ_OK;
+}
+
 laq_status laq_last_device_status(const laq_params* p, const void* ws, size_t ws_bytes,
                                   void* cuda_stream) {
   Dims d;
@@ -270,6 +338,11 @@ laq_status laq_last_device_status(const laq_params* p, const void* ws, size_t ws
   if (cudaMemcpy(hdr, ws, sizeof hdr, cudaMemcpyDeviceToHost) != cudaSuccess) return LAQ_ERR_CUDA;
   if (hdr[HDR_STATUS] == 0) return LAQ_OK;
   return hdr[HDR_STATUS] == LAQ_ERR_TIMEOUT ? LAQ_ERR_TIMEOUT : LAQ_ERR_INTERNAL;
+}
+
+void laq_set_stage_events(void* score_begin, void* score_end) {
+  g_ev_begin = (cudaEvent_t)score_begin;
+  g_ev_end = (cudaEvent_t)score_end;
 }
 
 int laq_last_launch_count(void) { return g_last_launches; }

@@ -15,6 +15,7 @@ struct Dims {
   int Ls, Kb;   // scored positions, selected slots
   int64_t U;    // units
   float scale;  // softmax scale
+  int tiles_per_task, sched_lag_units;  // caller's scheduling knobs (0 = automatic)
 };
 
 // Workspace layout (all offsets in bytes from the 256-byte aligned base).
