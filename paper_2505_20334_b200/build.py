@@ -34,7 +34,10 @@ def _deps_mtime():
     return max(os.path.getmtime(f) for f in files)
 
 
-def build_liblaq(force: bool = False, verbose: bool = False) -> str:
+def build_liblaq(force: bool = False, verbose: bool = False, defines=()) -> str:
+    """Compiles liblaq.so if it is missing or older than its sources. `defines` are extra
+    ``-DNAME=VALUE`` strings for tuning builds (they force a rebuild)."""
+    force = force or bool(defines)
     if not force and os.path.exists(LIB_PATH) and os.path.getmtime(LIB_PATH) >= _deps_mtime():
         return LIB_PATH
     os.makedirs(OBJ_DIR, exist_ok=True)
@@ -43,7 +46,7 @@ def build_liblaq(force: bool = False, verbose: bool = False) -> str:
 
     def compile_one(src):
         obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
-        cmd = [nvcc, *NVCC_FLAGS, *extra, "-c", src, "-o", obj]
+        cmd = [nvcc, *NVCC_FLAGS, *extra, *defines, "-c", src, "-o", obj]
         r = subprocess.run(cmd, capture_output=True, text=True)
         return obj, r
 
@@ -64,4 +67,5 @@ def build_liblaq(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build_liblaq(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_liblaq(force="--force" in sys.argv, verbose="-v" in sys.argv,
+                       defines=[a for a in sys.argv[1:] if a.startswith("-D")]))

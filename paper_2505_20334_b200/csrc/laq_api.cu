@@ -71,8 +71,9 @@ static laq_status check_strides_vo(const laq_params* p, bool need_v) {
 
 int choose_tiles_per_task(const Dims& d) {
   const int n_tiles = (d.L + TILE_KEYS - 1) / TILE_KEYS;
-  int t = d.tiles_per_task > 0 ? d.tiles_per_task : (n_tiles + 63) / 64;
-  if (d.tiles_per_task <= 0 && t < 4) t = 4;
+  // default: at most 32 tasks per unit and sweep, and at least 8 tiles per task
+  int t = d.tiles_per_task > 0 ? d.tiles_per_task : (n_tiles + 31) / 32;
+  if (d.tiles_per_task <= 0 && t < 8) t = 8;
   if (t > n_tiles) t = n_tiles;
   return t;
 }
@@ -80,15 +81,13 @@ int choose_tiles_per_task(const Dims& d) {
 void plan_workspace(const Dims& d, int tiles_per_task, Workspace* w) {
   const int n_tiles = (d.L + TILE_KEYS - 1) / TILE_KEYS;
   const int n_tasks = (n_tiles + tiles_per_task - 1) / tiles_per_task;
-  w->n_part = 2 * n_tasks;
+  w->n_part = n_tasks;
   w->M_pad = (d.M + 31) / 32 * 32;
   w->L_pad = n_tiles * TILE_KEYS;
   size_t off = 0;
   w->off_hdr = off;
   off = align_up(off + HDR_WORDS * sizeof(int32_t), 256);
   w->off_cnt = off;
-  off = align_up(off + (size_t)d.U * sizeof(int32_t), 256);
-  w->off_rdy = off;
   off = align_up(off + (size_t)d.U * sizeof(int32_t), 256);
   w->off_part = off;
   off = align_up(off + (size_t)d.U * w->n_part * w->M_pad * sizeof(float2), 256);
@@ -112,7 +111,7 @@ static thread_local cudaEvent_t g_ev_begin = nullptr, g_ev_end = nullptr;
 static laq_status run_scoring(const laq_params* p, const Dims& d, const Workspace& w,
                               const void* q, const void* k, char* ws, cudaStream_t stream,
                               int* launches) {
-  // header, unit counters and ready flags are contiguous: one clear
+  // header and unit counters are contiguous: one clear
   if (cudaMemsetAsync(ws + w.off_hdr, 0, w.off_part - w.off_hdr, stream) != cudaSuccess)
     return LAQ_ERR_CUDA;
   if (g_ev_begin && cudaEventRecord(g_ev_begin, stream) != cudaSuccess) return LAQ_ERR_CUDA;

@@ -21,15 +21,14 @@ struct Dims {
 // Workspace layout (all offsets in bytes from the 256-byte aligned base).
 //   header   : int32 words (see HDR_*), zeroed at the start of every scoring call
 //   unit_cnt : int32 [U]   partial row statistics delivered so far, zeroed per call
-//   unit_rdy : int32 [U]   1 once row_off of the unit is final, zeroed per call
-//   part     : float2 [U][n_part][M_pad]  partial (max, sum) in the log2 domain
-//   row_off  : float [U][M_pad]  b_r = log2e*scale*m_r + log2(l_r)
+//   part     : float2 [U][n_part][M_pad]  partial (max, sum) in the log2 domain, one per task
+//   row_off  : float [U][M_pad]  b_r = log2e*scale*m_r + log2(l_r) (CUDA-core path only)
 //   colsum   : float [U][L_pad]  c_j (step 3)
 //   pooled   : float [U][Ls]     p_j (step 4) when the caller gave no scores buffer
 //   idx      : int32 [U][B]      kept positions when the caller gave no idx buffer
 struct Workspace {
-  size_t off_hdr, off_cnt, off_rdy, off_part, off_rowoff, off_colsum, off_pooled, off_idx, total;
-  int n_part;  // partial-statistics slots per unit
+  size_t off_hdr, off_cnt, off_part, off_rowoff, off_colsum, off_pooled, off_idx, total;
+  int n_part;  // partial-statistics slots per unit = scoring tasks per unit and sweep
   int M_pad;   // rows padded to a multiple of 32
   int L_pad;   // L padded to a multiple of 128
 };

@@ -173,7 +173,7 @@ laq_status score_simt_launch(const laq_params& p, const Dims& d, const Workspace
   a.ks_head = p.k_stride_head;   a.ks_pos = p.k_stride_pos;
   a.Bt = d.Bt; a.Hkv = d.Hkv; a.G = d.G; a.W = d.W; a.D = d.D; a.L = d.L; a.M = d.M;
   a.M_pad = w.M_pad; a.n_part = w.n_part; a.L_pad = w.L_pad;
-  const int n_chunks = w.n_part / 2;
+  const int n_chunks = w.n_part;
   a.keys_per_chunk = (w.L_pad / TILE_KEYS + n_chunks - 1) / n_chunks * TILE_KEYS;
   a.scale_log2 = d.scale * kLog2e;
   a.part = (float2*)(ws + w.off_part);

@@ -9,29 +9,46 @@
 //                         and sums 2^(t[r][j] - b_r) over the rows r, b_r = m_r + log2(l_r).
 // Both sweeps read the same K tile layout (TMA, 128-byte swizzle) and differ only in which operand
 // the tile is. Tickets are ordered so that sweep 2 of a unit is handed out only after sweep 1 of
-// that unit (and of a few later units) has been handed out; a sweep-2 task waits, bounded, for the
-// unit's "statistics final" flag. A task therefore only ever depends on tasks with smaller tickets,
-// which running CTAs already hold, so the order is deadlock-free for any grid size. The second
-// sweep re-reads K while it is still resident in L2.
+// that unit (and of a few later units) has been handed out, so the second sweep re-reads K while
+// it is still resident in L2. A sweep-2 task needs the unit's row statistics, i.e. the partial
+// statistics of every sweep-1 task of the unit; those tasks have smaller tickets, which running
+// CTAs already hold, so the order is deadlock-free for any grid size. Every wait is bounded.
 //
-// Warp roles (384 threads): warp 0 = ticket fetch + TMA producer, warp 1 = tcgen05.mma issuer and
-// TMEM owner, warps 4-11 = two softmax warpgroups that alternate over the TMEM accumulator buffers.
+// Warp roles (384 threads):
+//   warp 0       ticket fetch + TMA producer (one lane)
+//   warp 1       tcgen05.mma issuer and TMEM owner (one lane)
+//   warp 2       statistics out: merges the two warpgroups' (max, sum) of a finished sweep-1 task,
+//                writes the task's partial to global memory and bumps the unit's counter
+//   warp 3       statistics in: for a sweep-2 task, waits for the unit's counter, merges the
+//                unit's partials into -b_r and hands them to the softmax warps in shared memory
+//   warps 4-11   two softmax warpgroups that alternate over the TMEM accumulator buffers
+// The softmax warps never wait on global memory: every global round trip of the statistics
+// exchange runs on the helper warps, ahead of or behind the tile pipeline.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
 #include "laq_internal.cuh"
+
+#ifndef LAQ_POLY_PAIRS_S1
+#define LAQ_POLY_PAIRS_S1 0  // of every 8 element pairs of sweep 1, this many use the FMA-pipe exp2
+#endif
+#ifndef LAQ_POLY_PAIRS_S2
+#define LAQ_POLY_PAIRS_S2 0  // same for sweep 2
+#endif
 
 namespace laq {
 namespace {
 
 constexpr int kThreads = 384;
 constexpr int kTaskSlots = 4;
-constexpr int kMaxKStages = 5;
+constexpr int kMaxKStages = 4;
 constexpr int kMaxBufs = 4;
+constexpr int kStatSlots = 2;
 constexpr uint32_t kKStageBytes = TILE_KEYS * 128 * 2;  // 128 keys x 128 dims x bf16
-constexpr uint32_t kCtlBytes = 3072;
+constexpr uint32_t kCtlBytes = 12288;
 constexpr long long kTimeoutCycles = 4000000000LL;  // ~2 s: every device-side wait gives up after this
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kTaskConsumers = 1 + 1 + 1 + 8;  // MMA lane, statistics-out warp, statistics-in warp, softmax warps
 
 struct TcArgs {
   int64_t U;
@@ -41,14 +58,13 @@ struct TcArgs {
   float scale_log2;
   int32_t* hdr;
   int32_t* cnt;
-  int32_t* rdy;
   float2* part;
-  float* row_off;
   float* colsum;
   int q_rows;     // rows allocated per 64-column half of a Q stage (128 or 256)
   int n_kstages;  // K stages in shared memory
   int tb_cols;    // TMEM columns per accumulator buffer (128 or 256)
   int n_bufs;     // accumulator buffers (4 or 2)
+  int use_hints;  // L2 eviction hints on the K loads
 };
 
 struct Task {
@@ -65,12 +81,16 @@ struct Ctl {
   uint64_t k_full[kMaxKStages], k_empty[kMaxKStages];
   uint64_t tmem_full[kMaxBufs], tmem_empty[kMaxBufs];
   uint64_t task_full[kTaskSlots], task_empty[kTaskSlots];
-  uint64_t wg_bar[2];
+  uint64_t stat_full[kStatSlots], stat_empty[kStatSlots];
+  uint64_t boff_full[kStatSlots], boff_empty[kStatSlots];
   Task tasks[kTaskSlots];
   uint32_t tmem_base;
   volatile int abort;
-  int wg_last[2];
-  float boff[2][256];  // per softmax warpgroup: b_r of the current sweep-2 task
+  uint32_t pad_[2];
+  // per finished sweep-1 task: (max, sum) of every row as seen by each softmax warpgroup
+  float2 stat[kStatSlots][2][256];
+  // per sweep-2 task: -b_r of every row (rows beyond M hold -1e30 so that they add nothing)
+  float nboff[kStatSlots][256];
 };
 static_assert(sizeof(Ctl) <= kCtlBytes, "control block too large");
 
@@ -99,12 +119,31 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
                                             int c0, int c1, int c2, int c3, int c4) {
   asm volatile(
       "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes "
       "[%0], [%1, {%3, %4, %5, %6, %7}], [%2];" ::"r"(dst),
       "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_5d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                                 int c0, int c1, int c2, int c3, int c4,
+                                                 uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4, %5, %6, %7}], [%2], %8;" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "l"(policy)
       : "memory");
 }
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
@@ -130,6 +169,11 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 // 32 consecutive fp32 columns of this thread's TMEM lane.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
   uint32_t* r = reinterpret_cast<uint32_t*>(v);
@@ -145,7 +189,8 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
       : "r"(taddr)
       : "memory");
 }
-// Waits for the loads above; the registers are named so that no use can move ahead of the wait.
+// Waits for every tcgen05.ld this thread has issued; the registers of the buffer about to be
+// used are named so that no use of them can move ahead of the wait.
 __device__ __forceinline__ void tmem_ld_wait(float* v) {
   uint32_t* r = reinterpret_cast<uint32_t*>(v);
   asm volatile("tcgen05.wait::ld.sync.aligned;"
@@ -173,6 +218,34 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
 __device__ __forceinline__ uint32_t instr_desc(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// ------------------------------------------------------------------ exponentials
+// 2^x on the FMA pipe for a pair of values: round-to-nearest split x = n + f, |f| <= 1/2, a
+// degree-3 polynomial for 2^f (max relative error 7.5e-5 over [-1/2, 1/2], fitted for this file)
+// and n added into the exponent field. Inputs below -126 are clamped (the result is then ~1e-38).
+__device__ __forceinline__ float2 exp2_fma_pair(float2 x) {
+  constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+  x.x = fmaxf(x.x, -126.0f);
+  x.y = fmaxf(x.y, -126.0f);
+  const float2 y = __fadd2_rn(x, make_float2(kMagic, kMagic));
+  const float2 n = __fadd2_rn(y, make_float2(-kMagic, -kMagic));
+  const float2 f = __ffma2_rn(n, make_float2(-1.0f, -1.0f), x);
+  float2 p = __ffma2_rn(make_float2(0.0551716685f, 0.0551716685f), f,
+                        make_float2(0.242611125f, 0.242611125f));
+  p = __ffma2_rn(p, f, make_float2(0.693260968f, 0.693260968f));
+  p = __ffma2_rn(p, f, make_float2(0.999928057f, 0.999928057f));
+  float2 r;
+  r.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(y.x) << 23));
+  r.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(y.y) << 23));
+  return r;
+}
+__device__ __forceinline__ float2 exp2_mufu_pair(float2 x) { return make_float2(ex2(x.x), ex2(x.y)); }
+
+// Pair p of a 32-column chunk goes to the FMA pipe if (p mod 8) < kPolyPairs, else to the MUFU.
+template <int kPolyPairs>
+__device__ __forceinline__ float2 exp2_pair(float2 x, int p) {
+  return ((p & 7) < kPolyPairs) ? exp2_fma_pair(x) : exp2_mufu_pair(x);
 }
 
 // ------------------------------------------------------------------ bounded waits
@@ -203,20 +276,6 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
   int v;
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
-}
-__device__ __forceinline__ void st_release(int32_t* p, int v) {
-  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-
-// Warpgroup barrier on an mbarrier (4 warp arrivals), bounded like every other wait.
-__device__ __forceinline__ bool wg_sync(const TcArgs& a, Ctl* ctl, int wg, uint32_t& phase,
-                                        int lane) {
-  __syncwarp();
-  const uint32_t bar = smem_u32(&ctl->wg_bar[wg]);
-  if (lane == 0) mbar_arrive(bar);
-  const bool ok = mbar_wait(a, ctl, bar, phase, 7);
-  phase ^= 1u;
-  return ok;
 }
 
 // Ticket -> task. Order: unit steps i = 0 .. U+lag-1; step i hands out the sweep-1 tasks of unit i
@@ -249,57 +308,135 @@ __device__ __forceinline__ void decode_ticket(const TcArgs& a, uint32_t t, Task&
   task.layer = (int)(unit / ((uint32_t)a.Hkv * (uint32_t)a.Bt));
 }
 
+// Every consumer warp reads the task ring the same way.
+__device__ __forceinline__ bool next_task(const TcArgs& a, Ctl* ctl, uint32_t& tk, int lane,
+                                          bool one_lane, int site, Task& task) {
+  const uint32_t slot = tk % kTaskSlots;
+  if (!mbar_wait(a, ctl, smem_u32(&ctl->task_full[slot]), (tk / kTaskSlots) & 1u, site)) return false;
+  task = ctl->tasks[slot];
+  if (!one_lane) __syncwarp();
+  if (lane == 0) mbar_arrive(smem_u32(&ctl->task_empty[slot]));
+  ++tk;
+  return true;
+}
+
+// Merges (max, sum) pairs in the log2 domain.
+__device__ __forceinline__ void merge_stat(float& m, float& l, float2 pr) {
+  const float mn = fmaxf(m, pr.x);
+  l = l * ex2(m - mn) + pr.y * ex2(pr.x - mn);
+  m = mn;
+}
+
 // ------------------------------------------------------------------ softmax-side tile work
-// Sweep 1: this thread owns query row `row`; 128 key columns of the tile, `valid` of them real.
-__device__ __forceinline__ void stats_tile(uint32_t taddr, int valid, float c, float& m, float& l) {
+// Sweep 1 keeps, per query row, a reference shift m and the sum l = sum_j 2^(t_j - m) of
+// t = c * s over the keys seen so far (log2 domain). m is only a reference, not the exact running
+// maximum: it moves up when a chunk holds a value more than kRebase above it, so the exponentials
+// of a chunk never wait for the chunk's own maximum. (m, l) pairs merge exactly as (max, sum)
+// pairs do, because only l * 2^m matters.
+constexpr float kRebase = 64.0f;
+
+// One full 32-column chunk of this thread's row.
+template <int kPolyPairs>
+__device__ __forceinline__ void stats_chunk(const float* v, float c, float& m, float& l) {
+  // largest raw logit of the chunk: four independent chains
+  float mx[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    mx[k] = max3(v[8 * k], v[8 * k + 1], v[8 * k + 2]);
+    mx[k] = max3(mx[k], v[8 * k + 3], v[8 * k + 4]);
+    mx[k] = max3(mx[k], v[8 * k + 5], v[8 * k + 6]);
+  }
+  const float t_max =
+      c * fmaxf(max3(mx[0], mx[1], mx[2]), max3(mx[3], max3(v[7], v[15], v[23]), v[31]));
+  const float2 c2 = make_float2(c, c), nm2 = make_float2(-m, -m);
+  float2 acc[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) acc[k] = make_float2(0.f, 0.f);
+#pragma unroll
+  for (int p = 0; p < 16; ++p) {
+    const float2 e =
+        exp2_pair<kPolyPairs>(__ffma2_rn(make_float2(v[2 * p], v[2 * p + 1]), c2, nm2), p);
+    acc[p & 3] = __fadd2_rn(acc[p & 3], e);
+  }
+  const float2 s2 = __fadd2_rn(__fadd2_rn(acc[0], acc[1]), __fadd2_rn(acc[2], acc[3]));
+  float sum = s2.x + s2.y;
+  if (__any_sync(0xffffffffu, t_max > m + kRebase)) {
+    // rare (first chunk of a task, or an outlier key): move the reference up and redo the chunk
+    const float m_new = fmaxf(m, t_max);
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+      s0 += ex2(fmaf(v[i], c, -m_new));
+      s1 += ex2(fmaf(v[i + 1], c, -m_new));
+    }
+    sum = s0 + s1;
+    l *= ex2(m - m_new);
+    m = m_new;
+  }
+  l += sum;
+}
+
+// A whole ragged tile (fewer than 128 real keys) of one row block, out of line: it only occurs
+// as the last tile of a unit whose prompt length is not a multiple of 128.
+__device__ __noinline__ float2 stats_tile_ragged(uint32_t taddr, int valid, float c, float m,
+                                                 float l) {
   float v[32];
-#pragma unroll 1
-  for (int c0 = 0; c0 < TILE_KEYS; c0 += 32) {
-    if (c0 >= valid) break;
-    tmem_ld32(taddr + c0, v);
+  for (int c0 = 0; c0 < valid; c0 += 32) {  // warp-uniform bounds
+    tmem_ld32(taddr + (uint32_t)c0, v);
     tmem_ld_wait(v);
     const int nv = valid - c0;
     float mx = v[0];
-    if (nv >= 32) {
 #pragma unroll
-      for (int i = 1; i < 32; ++i) mx = fmaxf(mx, v[i]);
-    } else {
-#pragma unroll
-      for (int i = 1; i < 32; ++i) mx = (i < nv) ? fmaxf(mx, v[i]) : mx;
-    }
+    for (int i = 1; i < 32; ++i) mx = (i < nv) ? fmaxf(mx, v[i]) : mx;
     const float m_new = fmaxf(m, mx * c);
     float sum = 0.f;
-    if (nv >= 32) {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) sum += ex2(fmaf(v[i], c, -m_new));
-    } else {
-#pragma unroll
-      for (int i = 0; i < 32; ++i) sum += (i < nv) ? ex2(fmaf(v[i], c, -m_new)) : 0.f;
-    }
-    l = l * ex2(m - m_new) + sum;
+    for (int i = 0; i < 32; ++i) sum += (i < nv) ? ex2(fmaf(v[i], c, -m_new)) : 0.f;
+    l = fmaf(l, ex2(m - m_new), sum);
     m = m_new;
+  }
+  return make_float2(m, l);
+}
+
+// Sweep 1, the 128 key columns of one row block of a full tile, with the TMEM load of the next
+// chunk in flight while a chunk is processed. If `release`, the accumulator buffer is handed back
+// to the MMA warp as soon as its last chunk is in registers.
+__device__ __forceinline__ void stats_block(uint32_t taddr, float c, float& m, float& l, float* va,
+                                            float* vb, bool release, uint32_t empty_bar, int lane) {
+  tmem_ld32(taddr, va);
+#pragma unroll 1
+  for (int h = 0; h < 2; ++h) {
+    tmem_ld_wait(va);
+    tmem_ld32(taddr + (uint32_t)h * 64u + 32u, vb);
+    stats_chunk<LAQ_POLY_PAIRS_S1>(va, c, m, l);
+    tmem_ld_wait(vb);
+    if (h == 0) {
+      tmem_ld32(taddr + 64u, va);
+    } else if (release) {
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_bar);
+    }
+    stats_chunk<LAQ_POLY_PAIRS_S1>(vb, c, m, l);
   }
 }
 
-// Sweep 2: this thread owns one key; sums the normalised weights over the M_pad row columns.
-__device__ __forceinline__ float colsum_tile(uint32_t taddr, int m_pad, float c, const float* boff) {
-  float v[32];
-  float acc = 0.f;
-#pragma unroll 1
-  for (int c0 = 0; c0 < m_pad; c0 += 32) {
-    tmem_ld32(taddr + c0, v);
-    tmem_ld_wait(v);
-    const float4* b4 = reinterpret_cast<const float4*>(boff + c0);
+// Sweep 2, one 32-column chunk (32 query rows) of this thread's key: adds 2^(c*s - b_r).
+// nb points at -b_r of the chunk's first row (shared memory, 16-byte aligned).
+template <int kPolyPairs>
+__device__ __forceinline__ void colsum_chunk(const float* v, float c, const float* nb, float2* acc) {
+  const float2 c2 = make_float2(c, c);
+  const float4* nb4 = reinterpret_cast<const float4*>(nb);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float4 bb = b4[i];
-      acc += ex2(fmaf(v[4 * i + 0], c, -bb.x));
-      acc += ex2(fmaf(v[4 * i + 1], c, -bb.y));
-      acc += ex2(fmaf(v[4 * i + 2], c, -bb.z));
-      acc += ex2(fmaf(v[4 * i + 3], c, -bb.w));
-    }
+  for (int i = 0; i < 8; ++i) {
+    const float4 bb = nb4[i];
+    const float2 e0 = exp2_pair<kPolyPairs>(
+        __ffma2_rn(make_float2(v[4 * i], v[4 * i + 1]), c2, make_float2(bb.x, bb.y)), 2 * i);
+    const float2 e1 = exp2_pair<kPolyPairs>(
+        __ffma2_rn(make_float2(v[4 * i + 2], v[4 * i + 3]), c2, make_float2(bb.z, bb.w)), 2 * i + 1);
+    acc[(2 * i) & 3] = __fadd2_rn(acc[(2 * i) & 3], e0);
+    acc[(2 * i + 1) & 3] = __fadd2_rn(acc[(2 * i + 1) & 3], e1);
   }
-  return acc;
 }
 
 // ------------------------------------------------------------------ the kernel
@@ -326,7 +463,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&ctl->q_full[i]), 1);
       mbar_init(smem_u32(&ctl->q_empty[i]), 1);
-      mbar_init(smem_u32(&ctl->wg_bar[i]), 4);
     }
     for (int i = 0; i < kMaxKStages; ++i) {
       mbar_init(smem_u32(&ctl->k_full[i]), 1);
@@ -338,10 +474,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
     }
     for (int i = 0; i < kTaskSlots; ++i) {
       mbar_init(smem_u32(&ctl->task_full[i]), 1);
-      mbar_init(smem_u32(&ctl->task_empty[i]), 9);
+      mbar_init(smem_u32(&ctl->task_empty[i]), kTaskConsumers);
+    }
+    for (int i = 0; i < kStatSlots; ++i) {
+      mbar_init(smem_u32(&ctl->stat_full[i]), 8);
+      mbar_init(smem_u32(&ctl->stat_empty[i]), 1);
+      mbar_init(smem_u32(&ctl->boff_full[i]), 1);
+      mbar_init(smem_u32(&ctl->boff_empty[i]), 8);
     }
     ctl->abort = 0;
-    ctl->wg_last[0] = ctl->wg_last[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   {
@@ -363,34 +504,22 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
   const uint32_t tmem_base = ctl->tmem_base;
 
   if (warp == 0) {
-    // ================= producer: tickets, dependency waits, TMA loads =================
+    // ================= producer: tickets and TMA loads =================
     if (lane == 0) {
       uint32_t kcount = 0, qcount = 0, tcount = 0;
+      const uint64_t pol_keep = l2_policy_evict_last(), pol_drop = l2_policy_evict_first();
+      unsigned int* ticket_ctr = reinterpret_cast<unsigned int*>(&a.hdr[HDR_TICKET]);
+      uint32_t next_ticket = atomicAdd(ticket_ctr, 1u);
       bool ok = true;
       while (ok) {
-        const uint32_t ticket = atomicAdd(reinterpret_cast<unsigned int*>(&a.hdr[HDR_TICKET]), 1u);
+        const uint32_t ticket = next_ticket;
         Task task;
         if (ticket >= a.total_tickets) {
           task.sweep = -1;
           task.unit = task.tile0 = task.n_tiles = task.chunk = task.layer = task.b = task.h = 0;
         } else {
           decode_ticket(a, ticket, task);
-        }
-        if (task.sweep == 1) {
-          // wait until the unit's row offsets are final
-          const int32_t* flag = &a.rdy[task.unit];
-          if (ld_acquire(flag) == 0) {
-            const long long t0 = clock64();
-            uint32_t spins = 0;
-            while (ld_acquire(flag) == 0) {
-              if ((++spins & 15u) == 0) {
-                if (ctl->abort) { ok = false; break; }
-                if (clock64() - t0 > kTimeoutCycles) { record_timeout(a, ctl, 1); ok = false; break; }
-              }
-              __nanosleep(64);
-            }
-          }
-          if (!ok) break;
+          next_ticket = atomicAdd(ticket_ctr, 1u);  // in flight while this task's loads are issued
         }
         const uint32_t slot = tcount % kTaskSlots;
         if (!mbar_wait(a, ctl, smem_u32(&ctl->task_empty[slot]), ((tcount / kTaskSlots) & 1u) ^ 1u, 2)) break;
@@ -410,6 +539,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
                       task.layer);
           ++qcount;
         }
+        // sweep 1 asks L2 to keep the tile for the second sweep, which then lets it go
+        const uint64_t pol = task.sweep == 0 ? pol_keep : pol_drop;
         for (int i = 0; i < task.n_tiles && ok; ++i) {
           const uint32_t s = kcount % (uint32_t)NS;
           if (!mbar_wait(a, ctl, smem_u32(&ctl->k_empty[s]), ((kcount / (uint32_t)NS) & 1u) ^ 1u, 4)) {
@@ -420,8 +551,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
           mbar_expect_tx(bar, kKStageBytes);
           const uint32_t dst = k_base + s * kKStageBytes;
           const int key0 = (task.tile0 + i) * TILE_KEYS;
-          tma_load_5d(dst, &tmap_k, bar, 0, key0, task.h, task.b, task.layer);
-          tma_load_5d(dst + kKStageBytes / 2, &tmap_k, bar, 64, key0, task.h, task.b, task.layer);
+          if (a.use_hints) {
+            tma_load_5d_hint(dst, &tmap_k, bar, 0, key0, task.h, task.b, task.layer, pol);
+            tma_load_5d_hint(dst + kKStageBytes / 2, &tmap_k, bar, 64, key0, task.h, task.b,
+                             task.layer, pol);
+          } else {
+            tma_load_5d(dst, &tmap_k, bar, 0, key0, task.h, task.b, task.layer);
+            tma_load_5d(dst + kKStageBytes / 2, &tmap_k, bar, 64, key0, task.h, task.b, task.layer);
+          }
           ++kcount;
         }
       }
@@ -440,11 +577,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       const int RB = (a.M + 127) / 128;
       bool ok = true;
       while (ok) {
-        const uint32_t slot = tk % kTaskSlots;
-        if (!mbar_wait(a, ctl, smem_u32(&ctl->task_full[slot]), (tk / kTaskSlots) & 1u, 10)) break;
-        const Task task = ctl->tasks[slot];
-        mbar_arrive(smem_u32(&ctl->task_empty[slot]));
-        ++tk;
+        Task task;
+        if (!next_task(a, ctl, tk, 0, true, 10, task)) break;
         if (task.sweep < 0) break;
         const uint32_t qs = qc & 1u;
         if (!mbar_wait(a, ctl, smem_u32(&ctl->q_full[qs]), (qc >> 1) & 1u, 11)) break;
@@ -488,6 +622,82 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         ++qc;
       }
     }
+  } else if (warp == 2) {
+    // ================= statistics out =================
+    uint32_t tk = 0, sc = 0;
+    while (true) {
+      Task task;
+      if (!next_task(a, ctl, tk, lane, false, 30, task)) break;
+      if (task.sweep < 0) break;
+      if (task.sweep != 0) continue;
+      const uint32_t s = sc % kStatSlots;
+      if (!mbar_wait(a, ctl, smem_u32(&ctl->stat_full[s]), (sc / kStatSlots) & 1u, 31)) break;
+      float2* dst = a.part + ((int64_t)task.unit * a.n_part + task.chunk) * a.M_pad;
+      for (int row = lane; row < a.M_pad; row += 32) {
+        float m = -1e30f, l = 0.f;
+        merge_stat(m, l, ctl->stat[s][0][row]);
+        merge_stat(m, l, ctl->stat[s][1][row]);
+        dst[row] = make_float2(m, l);
+      }
+      __threadfence();
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(smem_u32(&ctl->stat_empty[s]));
+        atomicAdd(&a.cnt[task.unit], 1);
+      }
+      ++sc;
+    }
+  } else if (warp == 3) {
+    // ================= statistics in =================
+    uint32_t tk = 0, sc = 0;
+    while (true) {
+      Task task;
+      if (!next_task(a, ctl, tk, lane, false, 40, task)) break;
+      if (task.sweep < 0) break;
+      if (task.sweep != 1) continue;
+      const uint32_t s = sc % kStatSlots;
+      if (!mbar_wait(a, ctl, smem_u32(&ctl->boff_empty[s]), ((sc / kStatSlots) & 1u) ^ 1u, 41)) break;
+      // every sweep-1 task of the unit must have delivered its partial
+      int ready = 1;
+      if (lane == 0) {
+        const int32_t* ctr = &a.cnt[task.unit];
+        if (ld_acquire(ctr) < a.tasks_per_unit) {
+          const long long t0 = clock64();
+          uint32_t spins = 0;
+          while (ld_acquire(ctr) < a.tasks_per_unit) {
+            if ((++spins & 15u) == 0) {
+              if (ctl->abort) { ready = 0; break; }
+              if (clock64() - t0 > kTimeoutCycles) { record_timeout(a, ctl, 42); ready = 0; break; }
+            }
+            __nanosleep(32);
+          }
+        }
+      }
+      ready = __shfl_sync(0xffffffffu, ready, 0);
+      if (!ready) break;
+      const float2* src = a.part + (int64_t)task.unit * a.n_part * a.M_pad;
+      for (int row = lane; row < 256; row += 32) {
+        float nb = -1e30f;
+        if (row < a.M) {
+          float m = -1e30f, l = 0.f;
+          const float2* pp = src + row;
+          int c0 = 0;
+          for (; c0 + 16 <= a.tasks_per_unit; c0 += 16) {
+            float2 pr[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pr[i] = __ldcg(pp + (int64_t)(c0 + i) * a.M_pad);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) merge_stat(m, l, pr[i]);
+          }
+          for (; c0 < a.tasks_per_unit; ++c0) merge_stat(m, l, __ldcg(pp + (int64_t)c0 * a.M_pad));
+          nb = -(m + log2f(l));
+        }
+        ctl->nboff[s][row] = nb;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctl->boff_full[s]));
+      ++sc;
+    }
   } else if (warp >= 4) {
     // ================= softmax warpgroups =================
     const int wg = (warp - 4) >> 2;
@@ -496,25 +706,20 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const float c = a.scale_log2;
     const int RB = (a.M + 127) / 128;
-    uint32_t tc = 0, tk = 0, wg_phase = 0;
-    float* boff = ctl->boff[wg];
+    const int n_chunks2 = a.M_pad / 32;
+    uint32_t tc = 0, tk = 0, s1c = 0, s2c = 0;
     bool ok = true;
     while (ok) {
-      const uint32_t slot = tk % kTaskSlots;
-      if (!mbar_wait(a, ctl, smem_u32(&ctl->task_full[slot]), (tk / kTaskSlots) & 1u, 20)) break;
-      const Task task = ctl->tasks[slot];
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&ctl->task_empty[slot]));
-      ++tk;
+      Task task;
+      if (!next_task(a, ctl, tk, lane, false, 20, task)) break;
       if (task.sweep < 0) break;
       const int64_t u = task.unit;
       float m[2] = {-1e30f, -1e30f}, l[2] = {0.f, 0.f};
+      const float* nboff = nullptr;
       if (task.sweep == 1) {
-        // b_r of this unit into the warpgroup's shared array (after the previous task's readers)
-        if (!wg_sync(a, ctl, wg, wg_phase, lane)) break;
-        for (int r = row_in_wg; r < 256; r += 128)
-          boff[r] = (r < a.M_pad) ? __ldcg(&a.row_off[u * a.M_pad + r]) : 1e30f;
-        if (!wg_sync(a, ctl, wg, wg_phase, lane)) break;
+        const uint32_t s = s2c % kStatSlots;
+        if (!mbar_wait(a, ctl, smem_u32(&ctl->boff_full[s]), (s2c / kStatSlots) & 1u, 22)) break;
+        nboff = ctl->nboff[s];
       }
       for (int i = 0; i < task.n_tiles; ++i, ++tc) {
         if ((int)(tc & 1u) != wg) continue;
@@ -527,64 +732,77 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         tc_fence_after();
         const int key0 = (task.tile0 + i) * TILE_KEYS;
         const uint32_t taddr = lane_addr + b * (uint32_t)a.tb_cols;
+        const uint32_t empty_bar = smem_u32(&ctl->tmem_empty[b]);
+        float va[32], vb[32];
         if (task.sweep == 0) {
           const int valid = min(TILE_KEYS, a.L - key0);
-          for (int rb = 0; rb < RB; ++rb) {
-            if (rb * 128 + quad * 32 < a.M)  // warp-uniform: skip row blocks beyond the unit's rows
-              stats_tile(taddr + (uint32_t)rb * 128u, valid, c, m[rb], l[rb]);
+          // row blocks beyond the unit's rows are skipped (warp-uniform)
+          const bool rows0 = quad * 32 < a.M, rows1 = RB == 2 && 128 + quad * 32 < a.M;
+          if (valid == TILE_KEYS) {
+            if (rows0) stats_block(taddr, c, m[0], l[0], va, vb, !rows1, empty_bar, lane);
+            if (rows1) stats_block(taddr + 128u, c, m[1], l[1], va, vb, true, empty_bar, lane);
+          } else {
+            if (rows0) {
+              const float2 r = stats_tile_ragged(taddr, valid, c, m[0], l[0]);
+              m[0] = r.x;
+              l[0] = r.y;
+            }
+            if (rows1) {
+              const float2 r = stats_tile_ragged(taddr + 128u, valid, c, m[1], l[1]);
+              m[1] = r.x;
+              l[1] = r.y;
+            }
+          }
+          if (valid != TILE_KEYS || (!rows0 && !rows1)) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_bar);
           }
         } else {
-          const float acc = colsum_tile(taddr, a.M_pad, c, boff);
+          float2 acc[4];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) acc[k] = make_float2(0.f, 0.f);
+          tmem_ld32(taddr, va);
+#pragma unroll 1
+          for (int ch = 0; ch < n_chunks2; ch += 2) {
+            tmem_ld_wait(va);
+            if (ch + 1 < n_chunks2) tmem_ld32(taddr + (uint32_t)(ch + 1) * 32u, vb);
+            if (ch + 1 >= n_chunks2) {
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(empty_bar);
+            }
+            colsum_chunk<LAQ_POLY_PAIRS_S2>(va, c, nboff + ch * 32, acc);
+            if (ch + 1 < n_chunks2) {
+              tmem_ld_wait(vb);
+              if (ch + 2 < n_chunks2) {
+                tmem_ld32(taddr + (uint32_t)(ch + 2) * 32u, va);
+              } else {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty_bar);
+              }
+              colsum_chunk<LAQ_POLY_PAIRS_S2>(vb, c, nboff + (ch + 1) * 32, acc);
+            }
+          }
+          const float2 s2 = __fadd2_rn(__fadd2_rn(acc[0], acc[1]), __fadd2_rn(acc[2], acc[3]));
           const int key = key0 + row_in_wg;
-          if (key < a.L) a.colsum[u * a.L_pad + key] = acc;
+          if (key < a.L) a.colsum[u * a.L_pad + key] = s2.x + s2.y;
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[b]));
       }
       if (!ok) break;
       if (task.sweep == 0) {
-        // deliver this warpgroup's partial statistics; the last delivery of the unit merges them
-        const int slot_p = task.chunk * 2 + wg;
-        for (int rb = 0; rb < RB; ++rb) {
-          const int row = rb * 128 + row_in_wg;
-          if (row < a.M_pad)
-            a.part[(u * a.n_part + slot_p) * a.M_pad + row] = make_float2(m[rb], l[rb]);
-        }
-        __threadfence();
-        if (!wg_sync(a, ctl, wg, wg_phase, lane)) break;
-        if (row_in_wg == 0) {
-          const int old = atomicAdd(&a.cnt[u], 1);
-          __threadfence();
-          ctl->wg_last[wg] = (old == a.n_part - 1);
-        }
-        if (!wg_sync(a, ctl, wg, wg_phase, lane)) break;
-        if (ctl->wg_last[wg]) {
-          for (int rb = 0; rb < RB; ++rb) {
-            const int row = rb * 128 + row_in_wg;
-            if (row < a.M_pad) {
-              float off = 1e30f;
-              if (row < a.M) {
-                float mm = -1e30f, ll = 0.f;
-                const float2* pp = a.part + u * a.n_part * a.M_pad + row;
-                for (int s = 0; s < a.n_part; ++s) {
-                  const float2 pr = __ldcg(pp + (int64_t)s * a.M_pad);
-                  if (pr.x > mm) {
-                    ll = ll * ex2(mm - pr.x) + pr.y;
-                    mm = pr.x;
-                  } else {
-                    ll += pr.y * ex2(pr.x - mm);
-                  }
-                }
-                off = mm + log2f(ll);
-              }
-              a.row_off[u * a.M_pad + row] = off;
-            }
-          }
-          __threadfence();
-          if (!wg_sync(a, ctl, wg, wg_phase, lane)) break;
-          if (row_in_wg == 0) st_release(&a.rdy[u], 1);
-        }
+        // hand this warpgroup's statistics to the statistics-out warp
+        const uint32_t s = s1c % kStatSlots;
+        if (!mbar_wait(a, ctl, smem_u32(&ctl->stat_empty[s]), ((s1c / kStatSlots) & 1u) ^ 1u, 23)) break;
+        for (int rb = 0; rb < 2; ++rb) ctl->stat[s][wg][rb * 128 + row_in_wg] = make_float2(m[rb], l[rb]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctl->stat_full[s]));
+        ++s1c;
+      } else {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctl->boff_empty[s2c % kStatSlots]));
+        ++s2c;
       }
     }
   }
@@ -648,7 +866,7 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   a.Bt = d.Bt; a.Hkv = d.Hkv; a.G = d.G; a.W = d.W; a.L = d.L; a.M = d.M;
   a.M_pad = w.M_pad; a.n_part = w.n_part; a.L_pad = w.L_pad;
   a.n_tiles = w.L_pad / TILE_KEYS;
-  a.tasks_per_unit = w.n_part / 2;
+  a.tasks_per_unit = w.n_part;
   a.tiles_per_task = (a.n_tiles + a.tasks_per_unit - 1) / a.tasks_per_unit;
   // every chunk must hold at least one tile
   if ((a.tasks_per_unit - 1) * a.tiles_per_task >= a.n_tiles || d.W > 256 || d.G > 256)
@@ -668,15 +886,14 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   a.scale_log2 = d.scale * kLog2e;
   a.hdr = (int32_t*)(ws + w.off_hdr);
   a.cnt = (int32_t*)(ws + w.off_cnt);
-  a.rdy = (int32_t*)(ws + w.off_rdy);
   a.part = (float2*)(ws + w.off_part);
-  a.row_off = (float*)(ws + w.off_rowoff);
   a.colsum = (float*)(ws + w.off_colsum);
   const bool wide = d.M > 128;
   a.q_rows = wide ? 256 : 128;
-  a.n_kstages = wide ? 3 : 4;
+  a.n_kstages = wide ? 2 : 4;
   a.tb_cols = wide ? 256 : 128;
   a.n_bufs = wide ? 2 : 4;
+  a.use_hints = 1;
 
   CUtensorMap tmap_q, tmap_k;
   const uint64_t qdims[5] = {128, (uint64_t)d.W, (uint64_t)d.Hq, (uint64_t)d.Bt, (uint64_t)d.NL};
