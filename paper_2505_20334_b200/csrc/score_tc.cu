@@ -4,7 +4,7 @@
 // One persistent CTA per SM pulls tasks from a global ticket counter. A task is one sweep over a
 // chunk of consecutive 128-key tiles of one unit:
 //   sweep 1 (statistics)  S  = Q K^T  : rows = queries on the TMEM lanes, so every softmax thread
-//                         owns one query row and keeps its running max / sum (log2 domain);
+//                         owns one query row and keeps a reference shift and a sum (log2 domain);
 //   sweep 2 (column sums) S^T = K Q^T : rows = keys on the TMEM lanes, so every thread owns one key
 //                         and sums 2^(t[r][j] - b_r) over the rows r, b_r = m_r + log2(l_r).
 // Both sweeps read the same K tile layout (TMA, 128-byte swizzle) and differ only in which operand
@@ -14,41 +14,45 @@
 // statistics of every sweep-1 task of the unit; those tasks have smaller tickets, which running
 // CTAs already hold, so the order is deadlock-free for any grid size. Every wait is bounded.
 //
-// Warp roles (384 threads):
+// Warp roles (640 threads):
 //   warp 0       ticket fetch + TMA producer (one lane)
 //   warp 1       tcgen05.mma issuer and TMEM owner (one lane)
-//   warp 2       statistics out: merges the two warpgroups' (max, sum) of a finished sweep-1 task,
+//   warp 2       statistics out: merges the warpgroups' (shift, sum) of a finished sweep-1 task,
 //                writes the task's partial to global memory and bumps the unit's counter
 //   warp 3       statistics in: for a sweep-2 task, waits for the unit's counter, merges the
 //                unit's partials into -b_r and hands them to the softmax warps in shared memory
-//   warps 4-11   two softmax warpgroups that alternate over the TMEM accumulator buffers
+//   warps 4-19   four softmax warpgroups in two pairs. Pair p takes the tiles t with t mod 2 == p;
+//                inside a pair the two warpgroups split the accumulator's columns in half, so a
+//                tile leaves its TMEM buffer quickly and the MMA warp can run several tiles ahead.
 // The softmax warps never wait on global memory: every global round trip of the statistics
 // exchange runs on the helper warps, ahead of or behind the tile pipeline.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
 #include "laq_internal.cuh"
+#include "softmax_math.cuh"
 
-#ifndef LAQ_POLY_PAIRS_S1
-#define LAQ_POLY_PAIRS_S1 0  // of every 8 element pairs of sweep 1, this many use the FMA-pipe exp2
-#endif
-#ifndef LAQ_POLY_PAIRS_S2
-#define LAQ_POLY_PAIRS_S2 0  // same for sweep 2
+#ifndef LAQ_PREFETCH_TILES
+#define LAQ_PREFETCH_TILES 4  // how many 128-key tiles the L2 prefetch of sweep 1 runs ahead of the loads
 #endif
 
 namespace laq {
 namespace {
 
-constexpr int kThreads = 384;
+using namespace laq::math;
+
+constexpr int kSoftmaxWgs = 4;
+constexpr int kSoftmaxWarps = 4 * kSoftmaxWgs;
+constexpr int kThreads = 128 + 128 * kSoftmaxWgs;
 constexpr int kTaskSlots = 4;
-constexpr int kMaxKStages = 4;
-constexpr int kMaxBufs = 4;
+constexpr int kMaxSlots = 4;  // K stages in shared memory = TMEM accumulator buffers
 constexpr int kStatSlots = 2;
 constexpr uint32_t kKStageBytes = TILE_KEYS * 128 * 2;  // 128 keys x 128 dims x bf16
-constexpr uint32_t kCtlBytes = 12288;
+constexpr uint32_t kCtlBytes = 22528;
 constexpr long long kTimeoutCycles = 4000000000LL;  // ~2 s: every device-side wait gives up after this
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kTaskConsumers = 1 + 1 + 1 + 8;  // MMA lane, statistics-out warp, statistics-in warp, softmax warps
+// MMA lane, statistics-out warp, statistics-in warp, softmax warps
+constexpr int kTaskConsumers = 3 + kSoftmaxWarps;
 
 struct TcArgs {
   int64_t U;
@@ -60,11 +64,10 @@ struct TcArgs {
   int32_t* cnt;
   float2* part;
   float* colsum;
-  int q_rows;     // rows allocated per 64-column half of a Q stage (128 or 256)
-  int n_kstages;  // K stages in shared memory
-  int tb_cols;    // TMEM columns per accumulator buffer (128 or 256)
-  int n_bufs;     // accumulator buffers (4 or 2)
-  int use_hints;  // L2 eviction hints on the K loads
+  int q_rows;      // rows allocated per 64-column half of a Q stage (128 or 256)
+  int n_slots;     // K stages = accumulator buffers (4, or 2 when a buffer takes 256 columns)
+  int slot_shift;  // log2(n_slots)
+  int tb_cols;     // TMEM columns per accumulator buffer (128 or 256)
 };
 
 struct Task {
@@ -78,8 +81,11 @@ struct Task {
 // Control block at the start of dynamic shared memory.
 struct Ctl {
   uint64_t q_full[2], q_empty[2];
-  uint64_t k_full[kMaxKStages], k_empty[kMaxKStages];
-  uint64_t tmem_full[kMaxBufs], tmem_empty[kMaxBufs];
+  uint64_t k_full[kMaxSlots];
+  // Tile t uses K stage t mod n_slots and accumulator buffer t mod n_slots, so one barrier per
+  // slot tells the producer that the stage is free and the softmax warps that the logits are ready.
+  uint64_t mma_done[kMaxSlots];
+  uint64_t tmem_empty[kMaxSlots];
   uint64_t task_full[kTaskSlots], task_empty[kTaskSlots];
   uint64_t stat_full[kStatSlots], stat_empty[kStatSlots];
   uint64_t boff_full[kStatSlots], boff_empty[kStatSlots];
@@ -87,10 +93,12 @@ struct Ctl {
   uint32_t tmem_base;
   volatile int abort;
   uint32_t pad_[2];
-  // per finished sweep-1 task: (max, sum) of every row as seen by each softmax warpgroup
-  float2 stat[kStatSlots][2][256];
+  // per finished sweep-1 task: (shift, sum) of every row as seen by each softmax warpgroup
+  float2 stat[kStatSlots][kSoftmaxWgs][256];
   // per sweep-2 task: -b_r of every row (rows beyond M hold -1e30 so that they add nothing)
   float nboff[kStatSlots][256];
+  // the same offsets prepared for the clamped FMA-pipe exponential: 1/2 - b_r/252
+  float nbsat[kStatSlots][256];
 };
 static_assert(sizeof(Ctl) <= kCtlBytes, "control block too large");
 
@@ -146,12 +154,22 @@ __device__ __forceinline__ void tma_load_5d_hint(uint32_t dst, const CUtensorMap
       "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "l"(policy)
       : "memory");
 }
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
-                                          uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void tma_prefetch_5d(const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                                int c4, uint64_t policy) {
   asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "cp.async.bulk.prefetch.tensor.5d.L2.global.tile.L2::cache_hint [%0, {%1, %2, %3, %4, %5}], %6;" ::"l"(map),
+      "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "l"(policy)
+      : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]; the two shared-memory descriptors are passed as (low, high) words.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo,
+                                          uint32_t desc_hi, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\n.reg .b64 da, db;\n"
+      "mov.b64 da, {%1, %3};\nmov.b64 db, {%2, %3};\n"
+      "setp.ne.b32 p, %5, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n}" ::"r"(d_tmem),
+      "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -163,16 +181,6 @@ __device__ __forceinline__ void tc_fence_before() {
 }
 __device__ __forceinline__ void tc_fence_after() {
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-}
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-  float d;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
 }
 // 32 consecutive fp32 columns of this thread's TMEM lane.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
@@ -203,49 +211,24 @@ __device__ __forceinline__ void tmem_ld_wait(float* v) {
                :
                : "memory");
 }
-
-// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, groups of
-// 8 rows 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);  // start address, bits [0,14)
-  d |= (uint64_t)1 << 16;                   // leading byte offset (not used by swizzled K-major)
-  d |= (uint64_t)(1024 >> 4) << 32;         // stride byte offset, bits [32,46)
-  d |= (uint64_t)1 << 46;                   // descriptor version of sm_100
-  d |= (uint64_t)2 << 61;                   // 128-byte swizzle
-  return d;
+// Adds to a global fp32 without returning a value.
+__device__ __forceinline__ void red_add(float* p, float v) {
+  asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
 }
+
+// Shared-memory matrix descriptor of a K-major operand with 128-byte swizzle, rows of 128 bytes
+// and groups of 8 rows 1024 bytes apart, split into its two words.
+// Low word: start address >> 4 in bits [0,14), leading byte offset (unused by swizzled K-major) in
+// bits [16,30). High word: stride byte offset 1024 >> 4 in bits [32,46), descriptor version 1 of
+// sm_100 at bit 46, 128-byte swizzle (2) at bits [61,64). Advancing the start address by `bytes`
+// (inside one shared-memory window below 256 KiB) is an add of bytes >> 4 to the low word.
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t addr) {
+  return ((addr & 0x3FFFFu) >> 4) | (1u << 16);
+}
+constexpr uint32_t kSmemDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
 __device__ __forceinline__ uint32_t instr_desc(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-
-// ------------------------------------------------------------------ exponentials
-// 2^x on the FMA pipe for a pair of values: round-to-nearest split x = n + f, |f| <= 1/2, a
-// degree-3 polynomial for 2^f (max relative error 7.5e-5 over [-1/2, 1/2], fitted for this file)
-// and n added into the exponent field. Inputs below -126 are clamped (the result is then ~1e-38).
-__device__ __forceinline__ float2 exp2_fma_pair(float2 x) {
-  constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
-  x.x = fmaxf(x.x, -126.0f);
-  x.y = fmaxf(x.y, -126.0f);
-  const float2 y = __fadd2_rn(x, make_float2(kMagic, kMagic));
-  const float2 n = __fadd2_rn(y, make_float2(-kMagic, -kMagic));
-  const float2 f = __ffma2_rn(n, make_float2(-1.0f, -1.0f), x);
-  float2 p = __ffma2_rn(make_float2(0.0551716685f, 0.0551716685f), f,
-                        make_float2(0.242611125f, 0.242611125f));
-  p = __ffma2_rn(p, f, make_float2(0.693260968f, 0.693260968f));
-  p = __ffma2_rn(p, f, make_float2(0.999928057f, 0.999928057f));
-  float2 r;
-  r.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(y.x) << 23));
-  r.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(y.y) << 23));
-  return r;
-}
-__device__ __forceinline__ float2 exp2_mufu_pair(float2 x) { return make_float2(ex2(x.x), ex2(x.y)); }
-
-// Pair p of a 32-column chunk goes to the FMA pipe if (p mod 8) < kPolyPairs, else to the MUFU.
-template <int kPolyPairs>
-__device__ __forceinline__ float2 exp2_pair(float2 x, int p) {
-  return ((p & 7) < kPolyPairs) ? exp2_fma_pair(x) : exp2_mufu_pair(x);
 }
 
 // ------------------------------------------------------------------ bounded waits
@@ -320,7 +303,7 @@ __device__ __forceinline__ bool next_task(const TcArgs& a, Ctl* ctl, uint32_t& t
   return true;
 }
 
-// Merges (max, sum) pairs in the log2 domain.
+// Merges (shift, sum) pairs in the log2 domain.
 __device__ __forceinline__ void merge_stat(float& m, float& l, float2 pr) {
   const float mn = fmaxf(m, pr.x);
   l = l * ex2(m - mn) + pr.y * ex2(pr.x - mn);
@@ -328,57 +311,16 @@ __device__ __forceinline__ void merge_stat(float& m, float& l, float2 pr) {
 }
 
 // ------------------------------------------------------------------ softmax-side tile work
-// Sweep 1 keeps, per query row, a reference shift m and the sum l = sum_j 2^(t_j - m) of
-// t = c * s over the keys seen so far (log2 domain). m is only a reference, not the exact running
-// maximum: it moves up when a chunk holds a value more than kRebase above it, so the exponentials
-// of a chunk never wait for the chunk's own maximum. (m, l) pairs merge exactly as (max, sum)
-// pairs do, because only l * 2^m matters.
-constexpr float kRebase = 64.0f;
-
-// One full 32-column chunk of this thread's row.
-template <int kPolyPairs>
-__device__ __forceinline__ void stats_chunk(const float* v, float c, float& m, float& l) {
-  // largest raw logit of the chunk: four independent chains
-  float mx[4];
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    mx[k] = max3(v[8 * k], v[8 * k + 1], v[8 * k + 2]);
-    mx[k] = max3(mx[k], v[8 * k + 3], v[8 * k + 4]);
-    mx[k] = max3(mx[k], v[8 * k + 5], v[8 * k + 6]);
-  }
-  const float t_max =
-      c * fmaxf(max3(mx[0], mx[1], mx[2]), max3(mx[3], max3(v[7], v[15], v[23]), v[31]));
-  const float2 c2 = make_float2(c, c), nm2 = make_float2(-m, -m);
-  float2 acc[4];
-#pragma unroll
-  for (int k = 0; k < 4; ++k) acc[k] = make_float2(0.f, 0.f);
-#pragma unroll
-  for (int p = 0; p < 16; ++p) {
-    const float2 e =
-        exp2_pair<kPolyPairs>(__ffma2_rn(make_float2(v[2 * p], v[2 * p + 1]), c2, nm2), p);
-    acc[p & 3] = __fadd2_rn(acc[p & 3], e);
-  }
-  const float2 s2 = __fadd2_rn(__fadd2_rn(acc[0], acc[1]), __fadd2_rn(acc[2], acc[3]));
-  float sum = s2.x + s2.y;
-  if (__any_sync(0xffffffffu, t_max > m + kRebase)) {
-    // rare (first chunk of a task, or an outlier key): move the reference up and redo the chunk
-    const float m_new = fmaxf(m, t_max);
-    float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-    for (int i = 0; i < 32; i += 2) {
-      s0 += ex2(fmaf(v[i], c, -m_new));
-      s1 += ex2(fmaf(v[i + 1], c, -m_new));
-    }
-    sum = s0 + s1;
-    l *= ex2(m - m_new);
-    m = m_new;
-  }
-  l += sum;
+// Hands a TMEM accumulator buffer back to the MMA warp once this warp has its share in registers.
+__device__ __forceinline__ void release_buffer(uint32_t empty_bar, int lane) {
+  tc_fence_before();
+  __syncwarp();
+  if (lane == 0) mbar_arrive(empty_bar);
 }
 
-// A whole ragged tile (fewer than 128 real keys) of one row block, out of line: it only occurs
-// as the last tile of a unit whose prompt length is not a multiple of 128.
-__device__ __noinline__ float2 stats_tile_ragged(uint32_t taddr, int valid, float c, float m,
+// Sweep 1, `valid` (< 64, possibly <= 0) real key columns starting at taddr, out of line: it only
+// occurs in the last tile of a unit whose prompt length is not a multiple of 128.
+__device__ __noinline__ float2 stats_cols_ragged(uint32_t taddr, int valid, float c, float m,
                                                  float l) {
   float v[32];
   for (int c0 = 0; c0 < valid; c0 += 32) {  // warp-uniform bounds
@@ -398,45 +340,17 @@ __device__ __noinline__ float2 stats_tile_ragged(uint32_t taddr, int valid, floa
   return make_float2(m, l);
 }
 
-// Sweep 1, the 128 key columns of one row block of a full tile, with the TMEM load of the next
-// chunk in flight while a chunk is processed. If `release`, the accumulator buffer is handed back
-// to the MMA warp as soon as its last chunk is in registers.
-__device__ __forceinline__ void stats_block(uint32_t taddr, float c, float& m, float& l, float* va,
-                                            float* vb, bool release, uint32_t empty_bar, int lane) {
-  tmem_ld32(taddr, va);
-#pragma unroll 1
-  for (int h = 0; h < 2; ++h) {
-    tmem_ld_wait(va);
-    tmem_ld32(taddr + (uint32_t)h * 64u + 32u, vb);
-    stats_chunk<LAQ_POLY_PAIRS_S1>(va, c, m, l);
-    tmem_ld_wait(vb);
-    if (h == 0) {
-      tmem_ld32(taddr + 64u, va);
-    } else if (release) {
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(empty_bar);
-    }
-    stats_chunk<LAQ_POLY_PAIRS_S1>(vb, c, m, l);
-  }
-}
-
-// Sweep 2, one 32-column chunk (32 query rows) of this thread's key: adds 2^(c*s - b_r).
-// nb points at -b_r of the chunk's first row (shared memory, 16-byte aligned).
-template <int kPolyPairs>
-__device__ __forceinline__ void colsum_chunk(const float* v, float c, const float* nb, float2* acc) {
-  const float2 c2 = make_float2(c, c);
-  const float4* nb4 = reinterpret_cast<const float4*>(nb);
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const float4 bb = nb4[i];
-    const float2 e0 = exp2_pair<kPolyPairs>(
-        __ffma2_rn(make_float2(v[4 * i], v[4 * i + 1]), c2, make_float2(bb.x, bb.y)), 2 * i);
-    const float2 e1 = exp2_pair<kPolyPairs>(
-        __ffma2_rn(make_float2(v[4 * i + 2], v[4 * i + 3]), c2, make_float2(bb.z, bb.w)), 2 * i + 1);
-    acc[(2 * i) & 3] = __fadd2_rn(acc[(2 * i) & 3], e0);
-    acc[(2 * i + 1) & 3] = __fadd2_rn(acc[(2 * i + 1) & 3], e1);
-  }
+// Sweep 1, this warpgroup's 64 key columns of one row block of a full tile. If `release`, the
+// accumulator buffer is handed back to the MMA warp as soon as the last chunk is in registers.
+__device__ __forceinline__ void stats_cols64(uint32_t taddr, float c, float& m, float& l, float* v,
+                                             bool release, uint32_t empty_bar, int lane) {
+  tmem_ld32(taddr, v);
+  tmem_ld_wait(v);
+  stats_chunk<LAQ_POLY_PAIRS_S1>(v, c, m, l);
+  tmem_ld32(taddr + 32u, v);
+  tmem_ld_wait(v);
+  if (release) release_buffer(empty_bar, lane);
+  stats_chunk<LAQ_POLY_PAIRS_S1>(v, c, m, l);
 }
 
 // ------------------------------------------------------------------ the kernel
@@ -450,7 +364,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
   const uint32_t q_base = smem_base + kCtlBytes;
   const uint32_t k_base = q_base + 2u * q_stage_bytes;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int NS = a.n_kstages, NB = a.n_bufs;
+  const uint32_t slot_mask = (uint32_t)a.n_slots - 1u;
 
   if ((smem_base & 1023u) != 0) {  // the swizzled stages need a 1024-byte aligned base
     if (threadIdx.x == 0 && atomicCAS(&a.hdr[HDR_STATUS], 0, (int)LAQ_ERR_INTERNAL) == 0)
@@ -464,23 +378,20 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       mbar_init(smem_u32(&ctl->q_full[i]), 1);
       mbar_init(smem_u32(&ctl->q_empty[i]), 1);
     }
-    for (int i = 0; i < kMaxKStages; ++i) {
+    for (int i = 0; i < kMaxSlots; ++i) {
       mbar_init(smem_u32(&ctl->k_full[i]), 1);
-      mbar_init(smem_u32(&ctl->k_empty[i]), 1);
-    }
-    for (int i = 0; i < kMaxBufs; ++i) {
-      mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
-      mbar_init(smem_u32(&ctl->tmem_empty[i]), 4);
+      mbar_init(smem_u32(&ctl->mma_done[i]), 1);
+      mbar_init(smem_u32(&ctl->tmem_empty[i]), 8);  // the 8 warps of one warpgroup pair
     }
     for (int i = 0; i < kTaskSlots; ++i) {
       mbar_init(smem_u32(&ctl->task_full[i]), 1);
       mbar_init(smem_u32(&ctl->task_empty[i]), kTaskConsumers);
     }
     for (int i = 0; i < kStatSlots; ++i) {
-      mbar_init(smem_u32(&ctl->stat_full[i]), 8);
+      mbar_init(smem_u32(&ctl->stat_full[i]), kSoftmaxWarps);
       mbar_init(smem_u32(&ctl->stat_empty[i]), 1);
       mbar_init(smem_u32(&ctl->boff_full[i]), 1);
-      mbar_init(smem_u32(&ctl->boff_empty[i]), 8);
+      mbar_init(smem_u32(&ctl->boff_empty[i]), kSoftmaxWarps);
     }
     ctl->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -509,18 +420,29 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       uint32_t kcount = 0, qcount = 0, tcount = 0;
       const uint64_t pol_keep = l2_policy_evict_last(), pol_drop = l2_policy_evict_first();
       unsigned int* ticket_ctr = reinterpret_cast<unsigned int*>(&a.hdr[HDR_TICKET]);
-      uint32_t next_ticket = atomicAdd(ticket_ctr, 1u);
+      const Task stop = {-1, 0, 0, 0, 0, 0, 0, 0};
+      // Asks L2 for tiles [first, first+count) of a sweep-1 task ahead of the loads into shared
+      // memory, so that the DRAM latency is not paid inside the shared-memory ring.
+      auto prefetch_tiles = [&](const Task& t, int first, int count) {
+        if (t.sweep != 0) return;
+        const int last = min(t.n_tiles, first + count);
+        for (int i = first; i < last; ++i) {
+          const int key0 = (t.tile0 + i) * TILE_KEYS;
+          tma_prefetch_5d(&tmap_k, 0, key0, t.h, t.b, t.layer, pol_keep);
+          tma_prefetch_5d(&tmap_k, 64, key0, t.h, t.b, t.layer, pol_keep);
+        }
+      };
+      Task task = stop;
+      {
+        const uint32_t t0 = atomicAdd(ticket_ctr, 1u);
+        if (t0 < a.total_tickets) decode_ticket(a, t0, task);
+      }
+      if (LAQ_PREFETCH_TILES > 0) prefetch_tiles(task, 0, LAQ_PREFETCH_TILES);
       bool ok = true;
       while (ok) {
-        const uint32_t ticket = next_ticket;
-        Task task;
-        if (ticket >= a.total_tickets) {
-          task.sweep = -1;
-          task.unit = task.tile0 = task.n_tiles = task.chunk = task.layer = task.b = task.h = 0;
-        } else {
-          decode_ticket(a, ticket, task);
-          next_ticket = atomicAdd(ticket_ctr, 1u);  // in flight while this task's loads are issued
-        }
+        // the next ticket is in flight while this task's loads are issued
+        uint32_t next_ticket = a.total_tickets;
+        if (task.sweep >= 0) next_ticket = atomicAdd(ticket_ctr, 1u);
         const uint32_t slot = tcount % kTaskSlots;
         if (!mbar_wait(a, ctl, smem_u32(&ctl->task_empty[slot]), ((tcount / kTaskSlots) & 1u) ^ 1u, 2)) break;
         ctl->tasks[slot] = task;
@@ -541,9 +463,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         }
         // sweep 1 asks L2 to keep the tile for the second sweep, which then lets it go
         const uint64_t pol = task.sweep == 0 ? pol_keep : pol_drop;
-        for (int i = 0; i < task.n_tiles && ok; ++i) {
-          const uint32_t s = kcount % (uint32_t)NS;
-          if (!mbar_wait(a, ctl, smem_u32(&ctl->k_empty[s]), ((kcount / (uint32_t)NS) & 1u) ^ 1u, 4)) {
+        Task next = stop;
+        bool next_known = false;
+        for (int i = 0; i < task.n_tiles; ++i) {
+          const uint32_t s = kcount & slot_mask;
+          // the stage is free once the MMAs of the tile that used it last have completed
+          if (!mbar_wait(a, ctl, smem_u32(&ctl->mma_done[s]), ((kcount >> a.slot_shift) & 1u) ^ 1u, 4)) {
             ok = false;
             break;
           }
@@ -551,16 +476,26 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
           mbar_expect_tx(bar, kKStageBytes);
           const uint32_t dst = k_base + s * kKStageBytes;
           const int key0 = (task.tile0 + i) * TILE_KEYS;
-          if (a.use_hints) {
-            tma_load_5d_hint(dst, &tmap_k, bar, 0, key0, task.h, task.b, task.layer, pol);
-            tma_load_5d_hint(dst + kKStageBytes / 2, &tmap_k, bar, 64, key0, task.h, task.b,
-                             task.layer, pol);
-          } else {
-            tma_load_5d(dst, &tmap_k, bar, 0, key0, task.h, task.b, task.layer);
-            tma_load_5d(dst + kKStageBytes / 2, &tmap_k, bar, 64, key0, task.h, task.b, task.layer);
-          }
+          tma_load_5d_hint(dst, &tmap_k, bar, 0, key0, task.h, task.b, task.layer, pol);
+          tma_load_5d_hint(dst + kKStageBytes / 2, &tmap_k, bar, 64, key0, task.h, task.b, task.layer,
+                           pol);
           ++kcount;
+          if (LAQ_PREFETCH_TILES > 0) {
+            // keep the L2 prefetch LAQ_PREFETCH_TILES tiles ahead, across the task boundary
+            const int ahead = i + LAQ_PREFETCH_TILES;
+            if (ahead < task.n_tiles) {
+              prefetch_tiles(task, ahead, 1);
+            } else {
+              if (!next_known) {
+                next_known = true;
+                if (next_ticket < a.total_tickets) decode_ticket(a, next_ticket, next);
+              }
+              prefetch_tiles(next, ahead - task.n_tiles, 1);
+            }
+          }
         }
+        if (!next_known && next_ticket < a.total_tickets) decode_ticket(a, next_ticket, next);
+        task = next;
       }
       if (ctl->abort) {
         // give loads that are still in flight time to land before the CTA exits
@@ -575,6 +510,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       const uint32_t idesc_s1 = instr_desc(128, TILE_KEYS);
       const uint32_t idesc_s2 = instr_desc(128, a.M_pad);
       const int RB = (a.M + 127) / 128;
+      const uint32_t q_half16 = (uint32_t)a.q_rows * 8u;  // (q_rows * 128 bytes) >> 4
+      const uint32_t k_lo0 = smem_desc_lo(k_base), q_lo0 = smem_desc_lo(q_base);
       bool ok = true;
       while (ok) {
         Task task;
@@ -582,40 +519,35 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         if (task.sweep < 0) break;
         const uint32_t qs = qc & 1u;
         if (!mbar_wait(a, ctl, smem_u32(&ctl->q_full[qs]), (qc >> 1) & 1u, 11)) break;
-        const uint32_t q_addr = q_base + qs * q_stage_bytes;
-        const uint32_t q_half = (uint32_t)a.q_rows * 128u;
-        for (int i = 0; i < task.n_tiles; ++i) {
-          const uint32_t s = tc % (uint32_t)NS, b = tc % (uint32_t)NB;
-          if (!mbar_wait(a, ctl, smem_u32(&ctl->k_full[s]), (tc / (uint32_t)NS) & 1u, 12) ||
-              !mbar_wait(a, ctl, smem_u32(&ctl->tmem_empty[b]), ((tc / (uint32_t)NB) & 1u) ^ 1u, 13)) {
+        const uint32_t q_lo = q_lo0 + qs * (q_stage_bytes >> 4);
+        for (int i = 0; i < task.n_tiles; ++i, ++tc) {
+          const uint32_t s = tc & slot_mask;
+          const uint32_t ph = (tc >> a.slot_shift) & 1u;
+          if (!mbar_wait(a, ctl, smem_u32(&ctl->k_full[s]), ph, 12) ||
+              !mbar_wait(a, ctl, smem_u32(&ctl->tmem_empty[s]), ph ^ 1u, 13)) {
             ok = false;
             break;
           }
           tc_fence_after();
-          const uint32_t k_addr = k_base + s * kKStageBytes;
-          const uint32_t d_tmem = tmem_base + b * (uint32_t)a.tb_cols;
+          const uint32_t k_lo = k_lo0 + s * (kKStageBytes >> 4);
+          const uint32_t d_tmem = tmem_base + s * (uint32_t)a.tb_cols;
+          // k-step kk covers dims [16 kk, 16 kk + 16): 32 bytes inside the 64-dim half (kk >> 2)
           if (task.sweep == 0) {
             for (int rb = 0; rb < RB; ++rb) {
 #pragma unroll
-              for (int kk = 0; kk < 8; ++kk) {
-                const uint32_t koff = (uint32_t)(kk & 3) * 32u;
-                const uint64_t da = smem_desc(q_addr + (kk >> 2) * q_half + (uint32_t)rb * 16384u + koff);
-                const uint64_t db = smem_desc(k_addr + (kk >> 2) * (kKStageBytes / 2) + koff);
-                umma_bf16(d_tmem + (uint32_t)rb * 128u, da, db, idesc_s1, kk > 0);
-              }
+              for (int kk = 0; kk < 8; ++kk)
+                umma_bf16(d_tmem + (uint32_t)rb * 128u,
+                          q_lo + (kk >> 2) * q_half16 + (uint32_t)rb * 1024u + (kk & 3) * 2u,
+                          k_lo + (kk >> 2) * (kKStageBytes >> 5) + (kk & 3) * 2u, kSmemDescHi,
+                          idesc_s1, kk > 0);
             }
           } else {
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-              const uint32_t koff = (uint32_t)(kk & 3) * 32u;
-              const uint64_t da = smem_desc(k_addr + (kk >> 2) * (kKStageBytes / 2) + koff);
-              const uint64_t db = smem_desc(q_addr + (kk >> 2) * q_half + koff);
-              umma_bf16(d_tmem, da, db, idesc_s2, kk > 0);
-            }
+            for (int kk = 0; kk < 8; ++kk)
+              umma_bf16(d_tmem, k_lo + (kk >> 2) * (kKStageBytes >> 5) + (kk & 3) * 2u,
+                        q_lo + (kk >> 2) * q_half16 + (kk & 3) * 2u, kSmemDescHi, idesc_s2, kk > 0);
           }
-          umma_commit(smem_u32(&ctl->k_empty[s]));
-          umma_commit(smem_u32(&ctl->tmem_full[b]));
-          ++tc;
+          umma_commit(smem_u32(&ctl->mma_done[s]));
         }
         if (!ok) break;
         umma_commit(smem_u32(&ctl->q_empty[qs]));
@@ -635,8 +567,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       float2* dst = a.part + ((int64_t)task.unit * a.n_part + task.chunk) * a.M_pad;
       for (int row = lane; row < a.M_pad; row += 32) {
         float m = -1e30f, l = 0.f;
-        merge_stat(m, l, ctl->stat[s][0][row]);
-        merge_stat(m, l, ctl->stat[s][1][row]);
+#pragma unroll
+        for (int g = 0; g < kSoftmaxWgs; ++g) merge_stat(m, l, ctl->stat[s][g][row]);
         dst[row] = make_float2(m, l);
       }
       __threadfence();
@@ -693,109 +625,112 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
           nb = -(m + log2f(l));
         }
         ctl->nboff[s][row] = nb;
+        ctl->nbsat[s][row] = fmaf(nb, kSatInv, 0.5f);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&ctl->boff_full[s]));
       ++sc;
     }
-  } else if (warp >= 4) {
+  } else {
     // ================= softmax warpgroups =================
     const int wg = (warp - 4) >> 2;
+    const int pair = wg >> 1, half = wg & 1;
     const int quad = warp & 3;
     const int row_in_wg = quad * 32 + lane;  // TMEM lane this thread reads
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const float c = a.scale_log2;
     const int RB = (a.M + 127) / 128;
+    // sweep 2: this warpgroup's share of the M_pad / 32 row chunks
     const int n_chunks2 = a.M_pad / 32;
-    uint32_t tc = 0, tk = 0, s1c = 0, s2c = 0;
+    const int ch_lo = half == 0 ? 0 : (n_chunks2 + 1) / 2;
+    const int ch_hi = half == 0 ? (n_chunks2 + 1) / 2 : n_chunks2;
+    const uint32_t col0 = 64u * (uint32_t)half;  // sweep 1: this warpgroup's 64 key columns
+    // Tiles are numbered through all tasks of this CTA; pair p owns tiles p, p + 2, ... A parity
+    // wait is sound because the previous use of a slot (tile t - n_slots) is never later than the
+    // pair's previous tile (t - 2).
+    uint32_t tc_base = 0, my_next = (uint32_t)pair, tk = 0, s1c = 0, s2c = 0;
     bool ok = true;
     while (ok) {
       Task task;
       if (!next_task(a, ctl, tk, lane, false, 20, task)) break;
       if (task.sweep < 0) break;
       const int64_t u = task.unit;
-      float m[2] = {-1e30f, -1e30f}, l[2] = {0.f, 0.f};
+      float m0 = -1e30f, l0 = 0.f, m1 = -1e30f, l1 = 0.f;
       const float* nboff = nullptr;
+      const float* nbsat = nullptr;
       if (task.sweep == 1) {
         const uint32_t s = s2c % kStatSlots;
         if (!mbar_wait(a, ctl, smem_u32(&ctl->boff_full[s]), (s2c / kStatSlots) & 1u, 22)) break;
         nboff = ctl->nboff[s];
+        nbsat = ctl->nbsat[s];
       }
-      for (int i = 0; i < task.n_tiles; ++i, ++tc) {
-        if ((int)(tc & 1u) != wg) continue;
-        const uint32_t b = tc % (uint32_t)NB;
-        if (!mbar_wait(a, ctl, smem_u32(&ctl->tmem_full[b]), (tc / (uint32_t)NB) & 1u, 21)) {
+      int i = (int)(my_next - tc_base);
+      for (; i < task.n_tiles; i += 2) {
+        const uint32_t tc = tc_base + (uint32_t)i;
+        const uint32_t s = tc & slot_mask;
+        if (!mbar_wait(a, ctl, smem_u32(&ctl->mma_done[s]), (tc >> a.slot_shift) & 1u, 21)) {
           ok = false;
           break;
         }
         __syncwarp();
         tc_fence_after();
         const int key0 = (task.tile0 + i) * TILE_KEYS;
-        const uint32_t taddr = lane_addr + b * (uint32_t)a.tb_cols;
-        const uint32_t empty_bar = smem_u32(&ctl->tmem_empty[b]);
-        float va[32], vb[32];
+        const uint32_t taddr = lane_addr + s * (uint32_t)a.tb_cols;
+        const uint32_t empty_bar = smem_u32(&ctl->tmem_empty[s]);
+        float v[32];
         if (task.sweep == 0) {
           const int valid = min(TILE_KEYS, a.L - key0);
           // row blocks beyond the unit's rows are skipped (warp-uniform)
           const bool rows0 = quad * 32 < a.M, rows1 = RB == 2 && 128 + quad * 32 < a.M;
           if (valid == TILE_KEYS) {
-            if (rows0) stats_block(taddr, c, m[0], l[0], va, vb, !rows1, empty_bar, lane);
-            if (rows1) stats_block(taddr + 128u, c, m[1], l[1], va, vb, true, empty_bar, lane);
+            if (rows0) stats_cols64(taddr + col0, c, m0, l0, v, !rows1, empty_bar, lane);
+            if (rows1) stats_cols64(taddr + 128u + col0, c, m1, l1, v, true, empty_bar, lane);
+            if (!rows0) release_buffer(empty_bar, lane);
           } else {
+            const int vh = min(64, valid - (int)col0);
             if (rows0) {
-              const float2 r = stats_tile_ragged(taddr, valid, c, m[0], l[0]);
-              m[0] = r.x;
-              l[0] = r.y;
+              const float2 r = stats_cols_ragged(taddr + col0, vh, c, m0, l0);
+              m0 = r.x;
+              l0 = r.y;
             }
             if (rows1) {
-              const float2 r = stats_tile_ragged(taddr + 128u, valid, c, m[1], l[1]);
-              m[1] = r.x;
-              l[1] = r.y;
+              const float2 r = stats_cols_ragged(taddr + 128u + col0, vh, c, m1, l1);
+              m1 = r.x;
+              l1 = r.y;
             }
-          }
-          if (valid != TILE_KEYS || (!rows0 && !rows1)) {
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty_bar);
+            release_buffer(empty_bar, lane);
           }
         } else {
           float2 acc[4];
 #pragma unroll
           for (int k = 0; k < 4; ++k) acc[k] = make_float2(0.f, 0.f);
-          tmem_ld32(taddr, va);
 #pragma unroll 1
-          for (int ch = 0; ch < n_chunks2; ch += 2) {
-            tmem_ld_wait(va);
-            if (ch + 1 < n_chunks2) tmem_ld32(taddr + (uint32_t)(ch + 1) * 32u, vb);
-            if (ch + 1 >= n_chunks2) {
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) mbar_arrive(empty_bar);
-            }
-            colsum_chunk<LAQ_POLY_PAIRS_S2>(va, c, nboff + ch * 32, acc);
-            if (ch + 1 < n_chunks2) {
-              tmem_ld_wait(vb);
-              if (ch + 2 < n_chunks2) {
-                tmem_ld32(taddr + (uint32_t)(ch + 2) * 32u, va);
-              } else {
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty_bar);
-              }
-              colsum_chunk<LAQ_POLY_PAIRS_S2>(vb, c, nboff + (ch + 1) * 32, acc);
-            }
+          for (int ch = ch_lo; ch < ch_hi; ++ch) {
+            tmem_ld32(taddr + (uint32_t)ch * 32u, v);
+            tmem_ld_wait(v);
+            if (ch + 1 == ch_hi) release_buffer(empty_bar, lane);
+            colsum_chunk<LAQ_POLY_PAIRS_S2>(v, c, nboff + ch * 32, nbsat + ch * 32, acc);
           }
-          const float2 s2 = __fadd2_rn(__fadd2_rn(acc[0], acc[1]), __fadd2_rn(acc[2], acc[3]));
-          const int key = key0 + row_in_wg;
-          if (key < a.L) a.colsum[u * a.L_pad + key] = s2.x + s2.y;
+          if (ch_lo == ch_hi) {
+            release_buffer(empty_bar, lane);
+          } else {
+            // The two warpgroups of the pair each add their rows' share into the zeroed column
+            // sum; with at most two addends the result does not depend on the order.
+            const float2 s2 = __fadd2_rn(__fadd2_rn(acc[0], acc[1]), __fadd2_rn(acc[2], acc[3]));
+            const int key = key0 + row_in_wg;
+            if (key < a.L) red_add(&a.colsum[u * a.L_pad + key], s2.x + s2.y);
+          }
         }
       }
       if (!ok) break;
+      my_next = tc_base + (uint32_t)i;
+      tc_base += (uint32_t)task.n_tiles;
       if (task.sweep == 0) {
         // hand this warpgroup's statistics to the statistics-out warp
         const uint32_t s = s1c % kStatSlots;
         if (!mbar_wait(a, ctl, smem_u32(&ctl->stat_empty[s]), ((s1c / kStatSlots) & 1u) ^ 1u, 23)) break;
-        for (int rb = 0; rb < 2; ++rb) ctl->stat[s][wg][rb * 128 + row_in_wg] = make_float2(m[rb], l[rb]);
+        ctl->stat[s][wg][row_in_wg] = make_float2(m0, l0);
+        ctl->stat[s][wg][128 + row_in_wg] = make_float2(m1, l1);
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctl->stat_full[s]));
         ++s1c;
@@ -890,10 +825,9 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   a.colsum = (float*)(ws + w.off_colsum);
   const bool wide = d.M > 128;
   a.q_rows = wide ? 256 : 128;
-  a.n_kstages = wide ? 2 : 4;
+  a.n_slots = wide ? 2 : 4;
+  a.slot_shift = wide ? 1 : 2;
   a.tb_cols = wide ? 256 : 128;
-  a.n_bufs = wide ? 2 : 4;
-  a.use_hints = 1;
 
   CUtensorMap tmap_q, tmap_k;
   const uint64_t qdims[5] = {128, (uint64_t)d.W, (uint64_t)d.Hq, (uint64_t)d.Bt, (uint64_t)d.NL};
@@ -905,9 +839,12 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   if (!make_map(&tmap_q, q, qdims, qstr, qbox) || !make_map(&tmap_k, k, kdims, kstr, kbox))
     return score_simt_launch(p, d, w, q, k, ws, stream, launches);  // layout TMA cannot describe
 
-  const size_t smem = kCtlBytes + 2u * (size_t)a.q_rows * 256u + (size_t)a.n_kstages * kKStageBytes;
+  const size_t smem = kCtlBytes + 2u * (size_t)a.q_rows * 256u + (size_t)a.n_slots * kKStageBytes;
   if (cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)smem) != cudaSuccess)
+    return LAQ_ERR_CUDA;
+  // the softmax warpgroups add their shares into the column sums, which therefore start at zero
+  if (cudaMemsetAsync(a.colsum, 0, (size_t)d.U * w.L_pad * sizeof(float), stream) != cudaSuccess)
     return LAQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.total_tickets < (uint32_t)sms ? a.total_tickets : (uint32_t)sms);
   score_tc_kernel<<<grid, kThreads, smem, stream>>>(tmap_q, tmap_k, a);
