@@ -14,9 +14,9 @@
 // statistics of every sweep-1 task of the unit; those tasks have smaller tickets, which running
 // CTAs already hold, so the order is deadlock-free for any grid size. Every wait is bounded.
 //
-// Warp roles (640 threads):
+// Warp roles (672 threads):
 //   warp 0       ticket fetch + TMA producer (one lane)
-//   warp 1       tcgen05.mma issuer and TMEM owner (one lane)
+//   warps 1, 20  tcgen05.mma issuers for alternate tiles (one lane each); warp 1 owns the TMEM
 //   warp 2       statistics out: merges the warpgroups' (shift, sum) of a finished sweep-1 task,
 //                writes the task's partial to global memory and bumps the unit's counter
 //   warp 3       statistics in: for a sweep-2 task, waits for the unit's counter, merges the
@@ -43,7 +43,8 @@ using namespace laq::math;
 
 constexpr int kSoftmaxWgs = 4;
 constexpr int kSoftmaxWarps = 4 * kSoftmaxWgs;
-constexpr int kThreads = 128 + 128 * kSoftmaxWgs;
+constexpr int kMmaWarpB = 4 + kSoftmaxWarps;  // index of the second MMA issuer's warp
+constexpr int kThreads = 32 * (kMmaWarpB + 1);
 constexpr int kTaskSlots = 4;
 constexpr int kMaxSlots = 4;  // K stages in shared memory = TMEM accumulator buffers
 constexpr int kStatSlots = 2;
@@ -51,8 +52,8 @@ constexpr uint32_t kKStageBytes = TILE_KEYS * 128 * 2;  // 128 keys x 128 dims x
 constexpr uint32_t kCtlBytes = 22528;
 constexpr long long kTimeoutCycles = 4000000000LL;  // ~2 s: every device-side wait gives up after this
 constexpr float kLog2e = 1.4426950408889634f;
-// MMA lane, statistics-out warp, statistics-in warp, softmax warps
-constexpr int kTaskConsumers = 3 + kSoftmaxWarps;
+// two MMA lanes, statistics-out warp, statistics-in warp, softmax warps
+constexpr int kTaskConsumers = 4 + kSoftmaxWarps;
 
 struct TcArgs {
   int64_t U;
@@ -376,7 +377,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&ctl->q_full[i]), 1);
-      mbar_init(smem_u32(&ctl->q_empty[i]), 1);
+      mbar_init(smem_u32(&ctl->q_empty[i]), 2);  // both MMA issuers
     }
     for (int i = 0; i < kMaxSlots; ++i) {
       mbar_init(smem_u32(&ctl->k_full[i]), 1);
@@ -503,10 +504,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         while (clock64() - t0 < 200000) __nanosleep(256);
       }
     }
-  } else if (warp == 1) {
-    // ================= MMA issuer =================
+  } else if (warp == 1 || warp == kMmaWarpB) {
+    // ================= MMA issuers =================
+    // Two lanes in two warps issue the tcgen05.mma of alternate tiles (issuer 0 those of the first
+    // softmax pair, issuer 1 those of the second), so that the scalar work and the barrier round
+    // trips of one tile overlap with the tensor-pipe time of the next. Tiles are independent:
+    // each has its own K stage, TMEM buffer and completion barrier.
     if (lane == 0) {
-      uint32_t tc = 0, qc = 0, tk = 0;
+      const uint32_t issuer = warp == 1 ? 0u : 1u;
+      uint32_t tc_base = 0, my_next = issuer, qc = 0, tk = 0;
       const uint32_t idesc_s1 = instr_desc(128, TILE_KEYS);
       const uint32_t idesc_s2 = instr_desc(128, a.M_pad);
       const int RB = (a.M + 127) / 128;
@@ -520,7 +526,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         const uint32_t qs = qc & 1u;
         if (!mbar_wait(a, ctl, smem_u32(&ctl->q_full[qs]), (qc >> 1) & 1u, 11)) break;
         const uint32_t q_lo = q_lo0 + qs * (q_stage_bytes >> 4);
-        for (int i = 0; i < task.n_tiles; ++i, ++tc) {
+        int i = (int)(my_next - tc_base);
+        for (; i < task.n_tiles; i += 2) {
+          const uint32_t tc = tc_base + (uint32_t)i;
           const uint32_t s = tc & slot_mask;
           const uint32_t ph = (tc >> a.slot_shift) & 1u;
           if (!mbar_wait(a, ctl, smem_u32(&ctl->k_full[s]), ph, 12) ||
@@ -550,6 +558,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
           umma_commit(smem_u32(&ctl->mma_done[s]));
         }
         if (!ok) break;
+        my_next = tc_base + (uint32_t)i;
+        tc_base += (uint32_t)task.n_tiles;
         umma_commit(smem_u32(&ctl->q_empty[qs]));
         ++qc;
       }
@@ -631,7 +641,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       if (lane == 0) mbar_arrive(smem_u32(&ctl->boff_full[s]));
       ++sc;
     }
-  } else {
+  } else if (warp >= 4) {
     // ================= softmax warpgroups =================
     const int wg = (warp - 4) >> 2;
     const int pair = wg >> 1, half = wg & 1;
