@@ -121,6 +121,36 @@ LAQ_API laq_status laq_score(const laq_params* p, const void* q, const void* k, 
                      void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * laq_score for callers that cannot allocate device memory. The paper has no counterpart to this
+ * entry point; it is an integration aid. It computes exactly what laq_score computes, but takes
+ * no workspace: its scratch is a fixed array of LAQ_STATIC_SCRATCH_BYTES bytes inside the library
+ * image (one copy on every GPU that loads the library, held until the process exits). It is meant
+ * for hosts that give all device memory to their own pool at start-up and may not call the
+ * driver's allocator afterwards -- an inference server whose allocator owns the GPU, a plugin
+ * that receives tensors and a stream but no allocator, a latency-critical loop that cannot take
+ * the device-wide synchronisation of an allocation. The call itself performs no allocation of
+ * any kind.
+ *   q, k, scores   as for laq_score (device pointers; scores dense [NL][Bt][Hkv][L-R], fp32)
+ * Limits and rules
+ *   - The problem's scratch (per-unit counters, per-task row statistics and one fp32 column sum
+ *     per key: roughly 4 bytes per cached key plus 8*M bytes per scoring task) must fit in
+ *     LAQ_STATIC_SCRATCH_BYTES; otherwise LAQ_ERR_WORKSPACE is returned and nothing is enqueued.
+ *     Larger problems can be scored in slices of layers with one call per slice.
+ *   - The first call on a device looks up the array's device address (with that device current)
+ *     and caches it; make that first call outside any stream capture.
+ *   - Every call uses the same array, which still holds the previous call's contents; the call
+ *     clears the parts that must start at zero. Two calls that overlap on the GPU (different
+ *     streams, or different host threads without ordering) race on it: order them.
+ *   - laq_last_device_status does not apply; a bounded device-side wait that runs out leaves the
+ *     scores undefined, as it does for laq_score.
+ * Errors: LAQ_ERR_INVALID_ARG, LAQ_ERR_UNSUPPORTED, LAQ_ERR_WORKSPACE (problem too large for the
+ * static scratch), LAQ_ERR_CUDA.
+ */
+#define LAQ_STATIC_SCRATCH_BYTES (8u * 1024u * 1024u)
+LAQ_API laq_status laq_score_static(const laq_params* p, const void* q, const void* k,
+                                    float* scores, void* cuda_stream);
+
+/*
  * Step 5 (Eq. 4's ArgSort(...)[:B]): per unit, the B-R positions of largest score, ties to the
  * lower position, then the retained tail.
  *   scores  device, fp32, dense [NL][Bt][Hkv][L-R], every value >= 0 and not NaN

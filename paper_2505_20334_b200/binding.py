@@ -27,6 +27,7 @@ EXPORTS = (
     "laq_params_dense_strides", "laq_workspace_bytes", "laq_score", "laq_select", "laq_compact",
     "laq_evict", "laq_last_device_status", "laq_last_launch_count", "laq_status_string",
     "laq_version", "laq_set_stage_events", "laq_host_staging_bytes", "laq_evict_host",
+    "laq_score_static",
 )
 
 
@@ -60,6 +61,8 @@ def _load() -> ctypes.CDLL:
     lib.laq_workspace_bytes.restype = sz
     lib.laq_score.argtypes = [pp, vp, vp, vp, vp, sz, vp]
     lib.laq_score.restype = ctypes.c_int
+    lib.laq_score_static.argtypes = [pp, vp, vp, vp, vp]
+    lib.laq_score_static.restype = ctypes.c_int
     lib.laq_select.argtypes = [pp, vp, vp, vp]
     lib.laq_select.restype = ctypes.c_int
     lib.laq_compact.argtypes = [pp, vp, vp, vp, vp, vp, vp]
@@ -148,6 +151,20 @@ def laq_score(p: LaqParams, q, k, scores, ws, stream=None, check=True) -> int:
     st = lib.laq_score(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(scores), wp, wn, _stream(stream))
     if check and st != LAQ_OK:
         raise LaqError(st, "laq_score")
+    return st
+
+
+STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
+
+
+def laq_score_static(p: LaqParams, q, k, scores, stream=None, check=True) -> int:
+    """``laq_score`` without a workspace argument, for callers that may not allocate device memory:
+    the scratch is a fixed ``STATIC_SCRATCH_BYTES`` array inside the library. Calls share that
+    array, so two of them must not overlap on the GPU; problems whose scratch does not fit are
+    refused with ``LAQ_ERR_WORKSPACE``."""
+    st = lib.laq_score_static(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(scores), _stream(stream))
+    if check and st != LAQ_OK:
+        raise LaqError(st, "laq_score_static")
     return st
 
 
