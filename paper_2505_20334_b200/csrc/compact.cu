@@ -1,6 +1,6 @@
 // Step 6: gathers the kept key/value rows into the dense compressed cache ("cache re-eviction
 // based on the given budget", Section 4.3). Pure 128-bit copies; each 16-byte vector of each
-// output row is one work item.
+// output row is one work item of a half-warp.
 #include "laq_internal.cuh"
 
 namespace laq {
@@ -20,25 +20,49 @@ struct CompactArgs {
   int64_t total;  // U * B * dv
 };
 
+// grid (row groups, units), block 256 threads = 16 half-warps. A half-warp copies one 256-byte
+// row (16 lanes x 16 bytes; wider rows take several steps), and every thread keeps kRowsInFlight
+// rows' loads in flight before it stores, so that the gather is limited by bandwidth and not by
+// the latency of one row.
+constexpr int kRowsInFlight = 4;
+constexpr int kRowsPerBlock = 16 * kRowsInFlight;
+
 __global__ void __launch_bounds__(256) compact_kernel(CompactArgs a) {
-  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < a.total; t += stride) {
-    const int c = (int)(t % a.dv);
-    const int64_t row = t / a.dv;  // u*B + slot
-    const int slot = (int)(row % a.B);
-    const int64_t u = row / a.B;
-    const int h = (int)(u % a.Hkv);
-    const int b = (int)((u / a.Hkv) % a.Bt);
-    const int64_t layer = u / ((int64_t)a.Hkv * a.Bt);
-    int32_t pos = a.idx[row];
-    pos = pos < 0 ? 0 : (pos >= a.L ? a.L - 1 : pos);  // never read outside the cache
-    const int64_t o = layer * a.os_layer + b * a.os_batch + h * a.os_head + slot * a.os_pos + c;
-    if (a.k_out)
-      __stcs(a.k_out + o, __ldcs(a.k + layer * a.ks_layer + b * a.ks_batch + h * a.ks_head +
-                                 pos * a.ks_pos + c));
-    if (a.v_out)
-      __stcs(a.v_out + o, __ldcs(a.v + layer * a.vs_layer + b * a.vs_batch + h * a.vs_head +
-                                 pos * a.vs_pos + c));
+  const int64_t u = blockIdx.y;
+  const int h = (int)(u % a.Hkv);
+  const int b = (int)((u / a.Hkv) % a.Bt);
+  const int64_t layer = u / ((int64_t)a.Hkv * a.Bt);
+  const int half_warp = threadIdx.x >> 4, c0 = threadIdx.x & 15;
+  const int slot0 = blockIdx.x * kRowsPerBlock + half_warp;
+  const int32_t* idx = a.idx + u * a.B;
+  const uint4* kbase = a.k + layer * a.ks_layer + b * a.ks_batch + h * a.ks_head;
+  const uint4* vbase = a.v + layer * a.vs_layer + b * a.vs_batch + h * a.vs_head;
+  const int64_t obase = layer * a.os_layer + b * a.os_batch + h * a.os_head;
+  int32_t pos[kRowsInFlight];
+#pragma unroll
+  for (int r = 0; r < kRowsInFlight; ++r) {
+    const int slot = slot0 + 16 * r;
+    int32_t p = slot < a.B ? idx[slot] : 0;
+    pos[r] = p < 0 ? 0 : (p >= a.L ? a.L - 1 : p);  // never read outside the cache
+  }
+  for (int c = c0; c < a.dv; c += 16) {
+    uint4 kv[kRowsInFlight], vv[kRowsInFlight];
+#pragma unroll
+    for (int r = 0; r < kRowsInFlight; ++r) {
+      if (slot0 + 16 * r < a.B) {
+        if (a.k_out) kv[r] = __ldcs(kbase + pos[r] * a.ks_pos + c);
+        if (a.v_out) vv[r] = __ldcs(vbase + pos[r] * a.vs_pos + c);
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < kRowsInFlight; ++r) {
+      const int slot = slot0 + 16 * r;
+      if (slot < a.B) {
+        const int64_t o = obase + slot * a.os_pos + c;
+        if (a.k_out) __stcs(a.k_out + o, kv[r]);
+        if (a.v_out) __stcs(a.v_out + o, vv[r]);
+      }
+    }
   }
 }
 
@@ -62,13 +86,9 @@ laq_status compact_launch(const laq_params& p, const Dims& d, const void* k, con
   a.os_head = p.o_stride_head / 8;   a.os_pos = p.o_stride_pos / 8;
   a.Bt = d.Bt; a.Hkv = d.Hkv; a.B = d.B; a.dv = d.D / 8; a.L = d.L;
   a.total = d.U * (int64_t)d.B * a.dv;
-  int dev = 0, sms = 148;
-  if (cudaGetDevice(&dev) == cudaSuccess)
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  int64_t blocks = (a.total + 255) / 256;
-  const int64_t cap = (int64_t)sms * 8;  // 8 resident blocks of 256 threads per SM
-  if (blocks > cap) blocks = cap;
-  compact_kernel<<<(unsigned)blocks, 256, 0, stream>>>(a);
+  if (d.U > 65535) return LAQ_ERR_UNSUPPORTED;
+  compact_kernel<<<dim3((unsigned)((d.B + kRowsPerBlock - 1) / kRowsPerBlock), (unsigned)d.U), 256, 0,
+                   stream>>>(a);
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;
 }

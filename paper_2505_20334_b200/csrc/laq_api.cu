@@ -254,12 +254,17 @@ laq_status laq_evict(const laq_params* p, const void* q, const void* k, const vo
   char* wsb = (char*)ws;
   int launches = 0;
   st = run_scoring(p, d, w, q, k, wsb, stream, &launches);
-  float* pooled = scores ? scores : (float*)(wsb + w.off_pooled);
-  if (st == LAQ_OK)
-    st = pool_launch(d, (const float*)(wsb + w.off_colsum), w.L_pad, pooled, stream, &launches);
   int32_t* idx_dev = idx ? idx : (int32_t*)(wsb + w.off_idx);
+  const float* colsum = (const float*)(wsb + w.off_colsum);
+  bool fused = false;
   if (st == LAQ_OK && (idx || k_out || v_out))
-    st = select_launch(d, pooled, idx_dev, stream, &launches);
+    st = pool_select_launch(d, colsum, w.L_pad, scores, idx_dev, stream, &launches, &fused);
+  if (st == LAQ_OK && !fused) {
+    float* pooled = scores ? scores : (float*)(wsb + w.off_pooled);
+    st = pool_launch(d, colsum, w.L_pad, pooled, stream, &launches);
+    if (st == LAQ_OK && (idx || k_out || v_out))
+      st = select_launch(d, pooled, idx_dev, stream, &launches);
+  }
   if (st == LAQ_OK && (k_out || v_out))
     st = compact_launch(*p, d, k, v, idx_dev, k_out, v_out, stream, &launches);
   g_last_launches = launches;

@@ -57,6 +57,10 @@ laq_status pool_launch(const Dims& d, const float* colsum, int L_pad, float* poo
 // Top-k (step 5) from pooled scores.
 laq_status select_launch(const Dims& d, const float* pooled, int32_t* idx, cudaStream_t stream,
                          int* launches);
+// Pool and top-k in one kernel when a unit's scores fit in shared memory (*done says whether it
+// ran; if not, nothing was enqueued). pooled_out may be NULL.
+laq_status pool_select_launch(const Dims& d, const float* colsum, int L_pad, float* pooled_out,
+                              int32_t* idx, cudaStream_t stream, int* launches, bool* done);
 // Gather (step 6).
 laq_status compact_launch(const laq_params& p, const Dims& d, const void* k, const void* v,
                           const int32_t* idx, void* k_out, void* v_out, cudaStream_t stream,

@@ -34,15 +34,10 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 // One block per unit. Four 8-bit radix passes find the key of the Kb-th largest score and how
 // many positions holding exactly that key are still needed; an ordered two-step compaction then
 // writes the kept positions in ascending order.
-__global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __restrict__ pooled,
-                                                             int32_t* __restrict__ idx, int Ls,
-                                                             int Kb, int R, int B) {
+__device__ __forceinline__ void select_unit(const float* p, int32_t* out, int Ls, int Kb, int R) {
   __shared__ uint32_t hist[256];
   __shared__ uint32_t s_prefix, s_need;
   __shared__ uint32_t s_gt[kSelWarps], s_eq[kSelWarps];
-  const int64_t u = blockIdx.x;
-  const float* p = pooled + u * (int64_t)Ls;
-  int32_t* out = idx + u * (int64_t)B;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   if (tid == 0) {
@@ -136,6 +131,40 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
   for (int t = tid; t < R; t += kSelThreads) out[Kb + t] = Ls + t;
 }
 
+// Step 5 alone: scores of unit blockIdx.x in global memory.
+__global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __restrict__ pooled,
+                                                             int32_t* __restrict__ idx, int Ls,
+                                                             int Kb, int R, int B) {
+  const int64_t u = blockIdx.x;
+  select_unit(pooled + u * (int64_t)Ls, idx + u * (int64_t)B, Ls, Kb, R);
+}
+
+// Steps 4 and 5 in one pass over the column sums: the block pools its unit's scores into shared
+// memory (and into `pooled_out` if the caller wants them), then selects from there, so that the
+// radix passes never go back to global memory. The pooling arithmetic is that of pool_kernel.
+__global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const float* __restrict__ colsum,
+                                                                  int L_pad, float* pooled_out,
+                                                                  int32_t* __restrict__ idx, int Ls,
+                                                                  int Kb, int R, int B, int kpool,
+                                                                  float inv_k) {
+  extern __shared__ float s_pooled[];
+  const int64_t u = blockIdx.x;
+  const float* c = colsum + u * (int64_t)L_pad;
+  const int h = kpool / 2;
+  for (int j = threadIdx.x; j < Ls; j += kSelThreads) {
+    float acc = 0.f;
+    for (int t = -h; t <= h; ++t) {
+      const int jj = j + t;
+      if (jj >= 0 && jj < Ls) acc += c[jj];
+    }
+    const float pj = acc * inv_k;
+    s_pooled[j] = pj;
+    if (pooled_out) pooled_out[u * (int64_t)Ls + j] = pj;
+  }
+  __syncthreads();
+  select_unit(s_pooled, idx + u * (int64_t)B, Ls, Kb, R);
+}
+
 }  // namespace
 
 laq_status pool_launch(const Dims& d, const float* colsum, int L_pad, float* pooled,
@@ -161,6 +190,21 @@ laq_status select_launch(const Dims& d, const float* pooled, int32_t* idx, cudaS
   if (d.U > 0x7fffffff) return LAQ_ERR_UNSUPPORTED;
   select_kernel<<<(unsigned)d.U, kSelThreads, 0, stream>>>(pooled, idx, d.Ls, d.Kb, d.R, d.B);
   *launches += 1;
+  return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;
+}
+
+laq_status pool_select_launch(const Dims& d, const float* colsum, int L_pad, float* pooled_out,
+                              int32_t* idx, cudaStream_t stream, int* launches, bool* done) {
+  *done = false;
+  const size_t smem = (size_t)d.Ls * sizeof(float);
+  if (smem > 200u * 1024u || d.U > 0x7fffffff) return LAQ_OK;  // the caller uses the two-kernel path
+  if (cudaFuncSetAttribute(pool_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)smem) != cudaSuccess)
+    return LAQ_ERR_CUDA;
+  pool_select_kernel<<<(unsigned)d.U, kSelThreads, smem, stream>>>(
+      colsum, L_pad, pooled_out, idx, d.Ls, d.Kb, d.R, d.B, d.kpool, 1.0f / (float)d.kpool);
+  *launches += 1;
+  *done = true;
   return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;
 }
 
