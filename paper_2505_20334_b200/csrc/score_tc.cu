@@ -825,7 +825,9 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
     return LAQ_ERR_CUDA;
   // sweep 2 trails sweep 1 by enough tasks that the statistics it needs are normally final
   int lag = d.sched_lag_units;
-  if (lag <= 0) lag = (3 * sms + 2 * a.tasks_per_unit - 1) / (2 * a.tasks_per_unit) + 1;
+  // (measured on B200: about 1.75 tickets per SM between the two sweeps of a unit is the smallest
+  // distance at which sweep-2 tasks rarely wait; a larger one only pushes K out of L2)
+  if (lag <= 0) lag = (7 * sms / 4 + 2 * a.tasks_per_unit - 1) / (2 * a.tasks_per_unit);
   if ((int64_t)lag > d.U) lag = (int)d.U;
   a.lag_units = lag;
   a.scale_log2 = d.scale * kLog2e;
