@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling)")
+    ap.add_argument("--prompt-len", type=int, default=0, help="override the prompt length (profiling)")
     ap.add_argument("--tiles-per-task", type=int, default=0)
     ap.add_argument("--lag-units", type=int, default=0)
     return ap.parse_args()
@@ -128,6 +130,10 @@ def workload(args):
     cfg = synth.CONFIGS[args.config]
     if args.layers:
         cfg = cfg.scaled(n_layers=args.layers)
+    if args.batch:
+        cfg = cfg.scaled(batch=args.batch)
+    if args.prompt_len:
+        cfg = cfg.scaled(prompt_len=args.prompt_len)
     return cfg
 
 
@@ -293,13 +299,11 @@ def main():
     score_ms = sum(a.elapsed_time(b) for a, b in ev) / K
     if laq.laq_last_device_status(p, ws) != laq.LAQ_OK:
         raise RuntimeError("laq_evict reported a device-side error")
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    from paper_2505_20334_b200 import multi
+
+    total_ms = multi.max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / K
-    tokens_per_step = cfg.batch * cfg.prompt_len * world
-    value = tokens_per_step / (ms_per_step * 1e-3)
+    value = multi.whole_job_tokens_per_s(cfg.batch * cfg.prompt_len, world, ms_per_step)
 
     peak, peak_src = measured_peaks()
     score_bytes, gather_bytes = algorithmic_bytes(cfg, B)
