@@ -165,6 +165,100 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const float* _
   select_unit(s_pooled, idx + u * (int64_t)B, Ls, Kb, R);
 }
 
+// Steps 4 and 5 for units of at most kRegItems * 1024 scored positions, with the unit's pooled
+// scores held in registers (kRegItems per thread) instead of memory. Warp w owns the contiguous
+// positions [1024 w, 1024 w + 1024), lane-strided, which is also the order the kept positions are
+// written in. The key of the Kb-th largest score is built bit by bit from the top: a candidate
+// bit stays set if at least Kb keys are >= the candidate; each step is 32 register compares per
+// thread, one warp reduction and one block barrier, with no atomics and no memory passes.
+// The pooling arithmetic is that of pool_kernel, so the scores are bit-identical to laq_score's.
+constexpr int kRegItems = 32;
+
+__global__ void __launch_bounds__(kSelThreads) pool_select_reg_kernel(
+    const float* __restrict__ colsum, int L_pad, float* pooled_out, int32_t* __restrict__ idx, int Ls,
+    int Kb, int R, int B, int kpool, float inv_k) {
+  __shared__ uint32_t s_cnt[2][kSelWarps];
+  __shared__ uint32_t s_gt[kSelWarps], s_eq[kSelWarps];
+  const int64_t u = blockIdx.x;
+  const float* c = colsum + u * (int64_t)L_pad;
+  int32_t* out = idx + u * (int64_t)B;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int base = warp * (kRegItems * 32) + lane;
+  const int h = kpool / 2;
+
+  uint32_t keys[kRegItems];
+#pragma unroll
+  for (int it = 0; it < kRegItems; ++it) {
+    const int j = base + it * 32;
+    uint32_t key = 0u;  // below the key of every real score
+    if (j < Ls) {
+      float acc = 0.f;
+      for (int t = -h; t <= h; ++t) {
+        const int jj = j + t;
+        if (jj >= 0 && jj < Ls) acc += c[jj];
+      }
+      const float pj = acc * inv_k;
+      if (pooled_out) pooled_out[u * (int64_t)Ls + j] = pj;
+      key = order_key(pj);
+    }
+    keys[it] = key;
+  }
+
+  // number of keys >= cand in the whole block (every warp computes the total)
+  int step = 0;
+  auto count_ge = [&](uint32_t cand) -> uint32_t {
+    uint32_t n = 0;
+#pragma unroll
+    for (int it = 0; it < kRegItems; ++it) n += keys[it] >= cand ? 1u : 0u;
+    n = __reduce_add_sync(0xffffffffu, n);
+    uint32_t* slot = s_cnt[step & 1];
+    ++step;
+    if (lane == 0) slot[warp] = n;
+    __syncthreads();
+    return __reduce_add_sync(0xffffffffu, slot[lane]);
+  };
+  uint32_t theta = 0u;
+#pragma unroll 1
+  for (int bit = 31; bit >= 0; --bit) {
+    const uint32_t cand = theta | (1u << bit);
+    if (count_ge(cand) >= (uint32_t)Kb) theta = cand;
+  }
+  // theta is the key of the Kb-th largest score; `need` positions holding exactly theta are kept
+  const uint32_t n_above = theta == 0xffffffffu ? 0u : count_ge(theta + 1u);
+  const uint32_t need = (uint32_t)Kb - n_above;
+
+  uint32_t n_gt = 0, n_eq = 0;
+#pragma unroll
+  for (int it = 0; it < kRegItems; ++it) {
+    n_gt += __popc(__ballot_sync(0xffffffffu, keys[it] > theta));
+    n_eq += __popc(__ballot_sync(0xffffffffu, keys[it] == theta));
+  }
+  if (lane == 0) {
+    s_gt[warp] = n_gt;
+    s_eq[warp] = n_eq;
+  }
+  __syncthreads();
+  uint32_t gt_run = 0, eq_run = 0;
+  for (int w = 0; w < warp; ++w) {
+    gt_run += s_gt[w];
+    eq_run += s_eq[w];
+  }
+  const uint32_t lt_mask = (1u << lane) - 1u;
+#pragma unroll
+  for (int it = 0; it < kRegItems; ++it) {
+    const bool gt = keys[it] > theta;
+    const bool eq = keys[it] == theta;
+    const uint32_t bg = __ballot_sync(0xffffffffu, gt);
+    const uint32_t be = __ballot_sync(0xffffffffu, eq);
+    const uint32_t gt_before = gt_run + __popc(bg & lt_mask);
+    const uint32_t eq_before = eq_run + __popc(be & lt_mask);
+    if (gt || (eq && eq_before < need)) out[gt_before + min(eq_before, need)] = base + it * 32;
+    gt_run += __popc(bg);
+    eq_run += __popc(be);
+  }
+  for (int t = tid; t < R; t += kSelThreads) out[Kb + t] = Ls + t;
+}
+
 }  // namespace
 
 laq_status pool_launch(const Dims& d, const float* colsum, int L_pad, float* pooled,
@@ -196,6 +290,14 @@ laq_status select_launch(const Dims& d, const float* pooled, int32_t* idx, cudaS
 laq_status pool_select_launch(const Dims& d, const float* colsum, int L_pad, float* pooled_out,
                               int32_t* idx, cudaStream_t stream, int* launches, bool* done) {
   *done = false;
+  if (d.U > 0x7fffffff) return LAQ_OK;
+  if (d.Ls <= kRegItems * kSelThreads) {
+    pool_select_reg_kernel<<<(unsigned)d.U, kSelThreads, 0, stream>>>(
+        colsum, L_pad, pooled_out, idx, d.Ls, d.Kb, d.R, d.B, d.kpool, 1.0f / (float)d.kpool);
+    *launches += 1;
+    *done = true;
+    return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;
+  }
   const size_t smem = (size_t)d.Ls * sizeof(float);
   if (smem > 200u * 1024u || d.U > 0x7fffffff) return LAQ_OK;  // the caller uses the two-kernel path
   if (cudaFuncSetAttribute(pool_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

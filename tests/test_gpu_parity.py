@@ -175,6 +175,28 @@ def test_edge_budgets_and_no_pooling(laq):
     compare_all_units(laq, q, k, v, 2, 15, 5)       # pool kernel wider than the scored range
 
 
+def test_evict_identical_keys_ties_go_to_lower_positions(laq):
+    # every key equal => all column sums equal; pooled interior equal, edges smaller: the kept
+    # set is [k/2, k/2 + Kb) by the tie rule, through the fused pool + select kernel
+    NL, Bt, Hq, Hkv, D, L, W, kernel, B = 1, 2, 4, 2, 128, 2500, 4, 7, 300
+    g = torch.Generator().manual_seed(31)
+    q = torch.randn((NL, Bt, Hq, W, D), generator=g).to(torch.bfloat16)
+    row = torch.randn((D,), generator=g).to(torch.bfloat16)
+    k = row.expand(NL, Bt, Hkv, L, D).contiguous()
+    v = torch.randn((NL, Bt, Hkv, L, D), generator=g).to(torch.bfloat16)
+    out = run_evict(laq, q, k, v, W, kernel, B)
+    idx = out["idx"].cpu().numpy()
+    Kb, Ls = B - W, L - W
+    want = np.concatenate([np.arange(kernel // 2, kernel // 2 + Kb), np.arange(Ls, L)])
+    got_scores = out["scores"].cpu().numpy()
+    for b in range(Bt):
+        for h in range(Hkv):
+            # equal inputs give bit-equal interior scores on the GPU as well
+            assert len(set(got_scores[0, b, h, kernel // 2: Ls - kernel // 2].tolist())) == 1
+            assert (idx[0, b, h] == want).all()
+            assert (idx[0, b, h] == orc.select(got_scores[0, b, h], L, W, B, sorted_variant=True)).all()
+
+
 def test_workspace_reuse_back_to_back(laq):
     q, k, v = rand_inputs(2, 1, 8, 2, 128, 1300, 8, seed=21)
     qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
