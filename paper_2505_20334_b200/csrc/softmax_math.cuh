@@ -8,7 +8,10 @@
 #include <stdint.h>
 
 #ifndef LAQ_POLY_PAIRS_S1
-#define LAQ_POLY_PAIRS_S1 2  // of every 8 element pairs of sweep 1, this many use the FMA-pipe exp2
+// Of every 8 element pairs, how many take the FMA-pipe exp2 instead of the MUFU. Alone, the
+// arithmetic is fastest at 2-3 of 8 (MUFU-bound below, FMA-bound above); inside the kernel on a
+// power-capped B200 0, 2 and 4 of 8 time within 1 % of each other.
+#define LAQ_POLY_PAIRS_S1 2
 #endif
 #ifndef LAQ_POLY_PAIRS_S2
 #define LAQ_POLY_PAIRS_S2 2  // same for sweep 2 (even)
