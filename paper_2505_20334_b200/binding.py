@@ -213,7 +213,8 @@ def laq_version() -> int:
 
 
 def evict(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, budget: int, pool_kernel: int = 7,
-          keep_tail: Optional[int] = None, want_scores: bool = False, ws=None, stream=None):
+          keep_tail: Optional[int] = None, want_scores: bool = False, ws=None, stream=None,
+          softmax_scale: float = 0.0):
     """Convenience call: allocates the outputs with torch and runs ``laq_evict``.
 
     q [NL,Bt,Hq,W,D], k and v [NL,Bt,Hkv,L,D], bf16 CUDA tensors. Returns a dict with 'k_out',
@@ -229,6 +230,7 @@ def evict(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, budget: int, pool_k
     idx = torch.empty((NL, Bt, Hkv, budget), dtype=torch.int32, device=k.device)
     scores = torch.empty((NL, Bt, Hkv, L - R), dtype=torch.float32, device=k.device) if want_scores else None
     p = params_for(q, k, R, pool_kernel, budget, v=v, out=k_out)
+    p.softmax_scale = softmax_scale  # 0 selects 1/sqrt(head_dim)
     if ws is None:
         ws = alloc_workspace(p, k.device)
     laq_evict(p, q, k, v, k_out, v_out, idx, scores, ws, stream)

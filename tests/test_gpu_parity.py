@@ -197,6 +197,36 @@ def test_evict_identical_keys_ties_go_to_lower_positions(laq):
             assert (idx[0, b, h] == orc.select(got_scores[0, b, h], L, W, B, sorted_variant=True)).all()
 
 
+def test_extreme_logits_and_late_maximum(laq):
+    # logits of +-hundreds: the running reference of sweep 1 has to move several times, also in the
+    # middle of a task, and sweep 2 sees probabilities far below the smallest fp32 normal
+    NL, Bt, Hq, Hkv, D, L, W, kernel, B = 1, 1, 8, 2, 128, 2304, 16, 7, 150
+    g = torch.Generator().manual_seed(404)
+    q = torch.randn((NL, Bt, Hq, W, D), generator=g).to(torch.bfloat16)
+    k = (torch.randn((NL, Bt, Hkv, L, D), generator=g) * 12.0).to(torch.bfloat16)
+    v = torch.randn((NL, Bt, Hkv, L, D), generator=g).to(torch.bfloat16)
+    # a key aligned with the mean query of each unit, very late in the prompt and very large
+    for h in range(Hkv):
+        qbar = q[0, 0, h * 4:(h + 1) * 4].float().mean(dim=(0, 1))
+        k[0, 0, h, 2100] = (qbar * 60.0).to(torch.bfloat16)
+    err, _ = compare_all_units(laq, q, k, v, W, kernel, B)
+    assert err < SCORE_RTOL
+
+
+def test_single_row_and_explicit_scale(laq):
+    # M = 1 (one query head per KV head, one lookahead query) and a caller-chosen softmax scale
+    NL, Bt, Hq, Hkv, D, L, W, kernel, B = 1, 2, 2, 2, 128, 700, 1, 3, 30
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=55)
+    scale = 0.05
+    out = laq.evict(q.cuda(), k.cuda(), v.cuda(), B, pool_kernel=kernel, keep_tail=W,
+                    want_scores=True, softmax_scale=scale)
+    ref = orc.evict(q, k, v, W, kernel, B, scale=scale)
+    assert score_rel_err(out["scores"].cpu().numpy(), ref["scores"]) <= SCORE_RTOL
+    # the default scale gives different scores, so the argument is really used
+    out2 = laq.evict(q.cuda(), k.cuda(), v.cuda(), B, pool_kernel=kernel, keep_tail=W, want_scores=True)
+    assert not torch.allclose(out["scores"], out2["scores"])
+
+
 def test_workspace_reuse_back_to_back(laq):
     q, k, v = rand_inputs(2, 1, 8, 2, 128, 1300, 8, seed=21)
     qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
