@@ -43,8 +43,25 @@ static double bf16_to_double(uint16_t h) {
  *   row_max  [G*W]     out (may be NULL): m_r
  *   row_sum  [G*W]     out (may be NULL): l_r
  */
+void laq_oracle_unit_colsum_local(const uint16_t* q, const uint16_t* k, int G, int W, int W_local,
+                                  int D, int L, double scale, double* c, double* row_max,
+                                  double* row_sum);
+
 void laq_oracle_unit_colsum(const uint16_t* q, const uint16_t* k, int G, int W, int D, int L,
                             double scale, double* c, double* row_max, double* row_sum) {
+  laq_oracle_unit_colsum_local(q, k, G, W, 0, D, L, scale, c, row_max, row_sum);
+}
+
+/*
+ * The same with the unified observation window of LAQ++ (Eq. 5: the sum runs over W u Q): the
+ * first W_local of each head's W queries are the queries of the last W_local prompt positions
+ * (query i sits at position L - W_local + i), the remaining W - W_local are lookahead queries.
+ * A local query attends causally, to the keys at positions <= its own; a lookahead query sees
+ * every prompt key. Keys a row cannot see get probability 0 from that row.
+ */
+void laq_oracle_unit_colsum_local(const uint16_t* q, const uint16_t* k, int G, int W, int W_local,
+                                  int D, int L, double scale, double* c, double* row_max,
+                                  double* row_sum) {
   const int M = G * W;
   double* s = (double*)malloc((size_t)L * sizeof(double));
   for (int j = 0; j < L; ++j) c[j] = 0.0;
@@ -56,14 +73,18 @@ void laq_oracle_unit_colsum(const uint16_t* q, const uint16_t* k, int G, int W, 
         acc += bf16_to_double(q[(size_t)r * D + d]) * bf16_to_double(k[(size_t)j * D + d]);
       s[j] = scale * acc;
     }
-    /* softmax over the L prompt keys */
+    /* keys this row can see: all of them for a lookahead query, positions <= its own for a
+     * local query (row r is query i = r mod W of head r / W) */
+    const int i = r % W;
+    const int vis = i < W_local ? L - W_local + i + 1 : L;
+    /* softmax over the visible prompt keys */
     double m = s[0];
-    for (int j = 1; j < L; ++j)
+    for (int j = 1; j < vis; ++j)
       if (s[j] > m) m = s[j];
     double l = 0.0;
-    for (int j = 0; j < L; ++j) l += exp(s[j] - m);
-    /* Eq. 4's sum over the window (and over the heads of the group) */
-    for (int j = 0; j < L; ++j) c[j] += exp(s[j] - m) / l;
+    for (int j = 0; j < vis; ++j) l += exp(s[j] - m);
+    /* Eq. 4 / Eq. 5: the sum over the window (and over the heads of the group) */
+    for (int j = 0; j < vis; ++j) c[j] += exp(s[j] - m) / l;
     if (row_max) row_max[r] = m;
     if (row_sum) row_sum[r] = l;
   }
@@ -159,8 +180,8 @@ void laq_oracle_compact(const uint16_t* src, const int32_t* idx, int B, int D, u
  * u = (layer*Bt + b)*Hkv + h; outputs of other units are left untouched.
  * Query head h*G+g belongs to KV head h. Returns the number of OpenMP threads used.
  */
-int laq_oracle_evict(const uint16_t* q, const uint16_t* k, const uint16_t* v, int NL, int Bt,
-                     int Hq, int Hkv, int D, int L, int W, int R, int kernel, int B,
+int laq_oracle_evict_local(const uint16_t* q, const uint16_t* k, const uint16_t* v, int NL, int Bt,
+                           int Hq, int Hkv, int D, int L, int W, int W_local, int R, int kernel, int B,
                      double scale, const int64_t* unit_list, int64_t n_units, double* scores,
                      double* colsum, int32_t* idx, uint16_t* k_out, uint16_t* v_out,
                      int fast_select) {
@@ -185,7 +206,7 @@ int laq_oracle_evict(const uint16_t* q, const uint16_t* k, const uint16_t* v, in
     const uint16_t* ku = k + u * (int64_t)L * D;
     double* c = (double*)malloc((size_t)L * sizeof(double));
     double* p = (double*)malloc((size_t)(Ls > 0 ? Ls : 1) * sizeof(double));
-    laq_oracle_unit_colsum(qu, ku, G, W, D, L, scale, c, NULL, NULL);
+    laq_oracle_unit_colsum_local(qu, ku, G, W, W_local, D, L, scale, c, NULL, NULL);
     laq_oracle_pool(c, Ls, kernel, p);
     if (colsum) memcpy(colsum + u * (int64_t)L, c, (size_t)L * sizeof(double));
     if (scores) memcpy(scores + u * (int64_t)Ls, p, (size_t)Ls * sizeof(double));
@@ -202,4 +223,13 @@ int laq_oracle_evict(const uint16_t* q, const uint16_t* k, const uint16_t* v, in
     free(p);
   }
   return threads;
+}
+
+int laq_oracle_evict(const uint16_t* q, const uint16_t* k, const uint16_t* v, int NL, int Bt,
+                     int Hq, int Hkv, int D, int L, int W, int R, int kernel, int B,
+                     double scale, const int64_t* unit_list, int64_t n_units, double* scores,
+                     double* colsum, int32_t* idx, uint16_t* k_out, uint16_t* v_out,
+                     int fast_select) {
+  return laq_oracle_evict_local(q, k, v, NL, Bt, Hq, Hkv, D, L, W, 0, R, kernel, B, scale, unit_list,
+                                n_units, scores, colsum, idx, k_out, v_out, fast_select);
 }

@@ -33,6 +33,8 @@ def _load():
         vp, i, d, i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_double, ctypes.c_int64
         lib.laq_oracle_unit_colsum.argtypes = [vp, vp, i, i, i, i, d, vp, vp, vp]
         lib.laq_oracle_unit_colsum.restype = None
+        lib.laq_oracle_unit_colsum_local.argtypes = [vp, vp, i, i, i, i, i, d, vp, vp, vp]
+        lib.laq_oracle_unit_colsum_local.restype = None
         lib.laq_oracle_pool.argtypes = [vp, i, i, vp]
         lib.laq_oracle_pool.restype = None
         lib.laq_oracle_select.argtypes = [vp, i, i, i, vp]
@@ -44,6 +46,9 @@ def _load():
         lib.laq_oracle_evict.argtypes = [vp, vp, vp, i, i, i, i, i, i, i, i, i, i, d, vp, i64,
                                          vp, vp, vp, vp, vp, i]
         lib.laq_oracle_evict.restype = i
+        lib.laq_oracle_evict_local.argtypes = [vp, vp, vp, i, i, i, i, i, i, i, i, i, i, i, d, vp, i64,
+                                               vp, vp, vp, vp, vp, i]
+        lib.laq_oracle_evict_local.restype = i
         _lib = lib
     return _lib
 
@@ -64,8 +69,10 @@ def _ptr(a):
     return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
 
 
-def unit_colsum(q, k, scale=None):
-    """q [G][W][D], k [L][D] bf16 -> (c [L], row_max [G*W], row_sum [G*W]) in fp64."""
+def unit_colsum(q, k, scale=None, local_window=0):
+    """q [G][W][D], k [L][D] bf16 -> (c [L], row_max [G*W], row_sum [G*W]) in fp64. With
+    `local_window` > 0 the first that many queries of each head are the causal queries of the last
+    prompt positions (the unified window of LAQ++, Eq. 5)."""
     q, k = _bits(q), _bits(k)
     G, W, D = q.shape
     L = k.shape[0]
@@ -74,7 +81,8 @@ def unit_colsum(q, k, scale=None):
     c = np.empty(L, np.float64)
     m = np.empty(G * W, np.float64)
     l = np.empty(G * W, np.float64)
-    _load().laq_oracle_unit_colsum(_ptr(q), _ptr(k), G, W, D, L, scale, _ptr(c), _ptr(m), _ptr(l))
+    _load().laq_oracle_unit_colsum_local(_ptr(q), _ptr(k), G, W, int(local_window), D, L, scale,
+                                         _ptr(c), _ptr(m), _ptr(l))
     return c, m, l
 
 
@@ -105,7 +113,7 @@ def compact(src, idx):
 
 
 def evict(q, k, v, R, kernel, B, scale=None, units=None, want_colsum=False, fast_select=True,
-          want_idx=True):
+          want_idx=True, local_window=0):
     """Whole step on dense tensors. q [NL][Bt][Hq][W][D], k/v [NL][Bt][Hkv][L][D] (bf16).
 
     Returns a dict with 'scores' [NL,Bt,Hkv,L-R] fp64, 'idx' [NL,Bt,Hkv,B] int32, 'k_out',
@@ -125,8 +133,8 @@ def evict(q, k, v, R, kernel, B, scale=None, units=None, want_colsum=False, fast
     k_out = np.zeros((NL, Bt, Hkv, B, D), np.uint16) if want_idx else None
     v_out = np.zeros((NL, Bt, Hkv, B, D), np.uint16) if (want_idx and v is not None) else None
     ul = None if units is None else np.ascontiguousarray(units, np.int64)
-    threads = _load().laq_oracle_evict(
-        _ptr(q), _ptr(k), _ptr(v), NL, Bt, Hq, Hkv, D, L, W, R, kernel, B, scale, _ptr(ul),
+    threads = _load().laq_oracle_evict_local(
+        _ptr(q), _ptr(k), _ptr(v), NL, Bt, Hq, Hkv, D, L, W, int(local_window), R, kernel, B, scale, _ptr(ul),
         0 if ul is None else ul.shape[0], _ptr(scores), _ptr(colsum), _ptr(idx), _ptr(k_out),
         _ptr(v_out), 1 if fast_select else 0)
     out = {"scores": scores, "idx": idx, "k_out": k_out, "v_out": v_out, "threads": threads}

@@ -296,3 +296,79 @@ def test_sink_and_needles_kept_when_budget_allows():
         kept = set(out["idx"][0, 0, h].tolist())
         assert 0 in kept
         assert set(inp["planted"]["needles"][0, 0, h].tolist()) <= kept
+
+
+# ---------------------------------------------------------------- LAQ++ unified window (Eq. 5)
+def _visible(i, W_local, L):
+    return L - W_local + i + 1 if i < W_local else L
+
+
+@pytest.mark.parametrize("G,W,Wl,D,L", [(1, 2, 1, 2, 4), (2, 4, 2, 4, 9), (2, 5, 5, 8, 12)])
+def test_local_window_bruteforce_causal_softmax(G, W, Wl, D, L):
+    q = rand_bf16((G, W, D), 900 + L)
+    k = rand_bf16((L, D), 901 + L)
+    scale = 0.37
+    c, m, l = orc.unit_colsum(q, k, scale=scale, local_window=Wl)
+    qf, kf = q.double().numpy(), k.double().numpy()
+    want = np.zeros(L)
+    for g in range(G):
+        for i in range(W):
+            vis = _visible(i, Wl, L)
+            logits = [scale * sum(qf[g, i, d] * kf[j, d] for d in range(D)) for j in range(vis)]
+            den = sum(math.exp(x) for x in logits)
+            for j in range(vis):
+                want[j] += math.exp(logits[j]) / den
+            r = g * W + i
+            assert m[r] == pytest.approx(max(logits), rel=1e-14, abs=1e-14)
+            assert l[r] == pytest.approx(sum(math.exp(x - max(logits)) for x in logits), rel=1e-13)
+    np.testing.assert_allclose(c, want, rtol=1e-13, atol=1e-15)
+
+
+def test_local_window_against_torch_masked_softmax():
+    G, W, Wl, D, L = 4, 16, 8, 32, 300
+    q, k = rand_bf16((G, W, D), 77), rand_bf16((L, D), 78)
+    scale = 1.0 / math.sqrt(D)
+    c, _, _ = orc.unit_colsum(q, k, local_window=Wl)
+    s = (q.double().reshape(G * W, D) @ k.double().T) * scale
+    mask = torch.zeros_like(s, dtype=torch.bool)
+    for r in range(G * W):
+        mask[r, _visible(r % W, Wl, L):] = True
+    want = torch.softmax(s.masked_fill(mask, -float("inf")), dim=-1).sum(0).numpy()
+    np.testing.assert_allclose(c, want, rtol=1e-12, atol=1e-15)
+    assert c.sum() == pytest.approx(G * W, rel=1e-12)       # every row still sums to one
+    # the last key is seen by the lookahead rows and by the last local query of each head only
+    assert c[L - 1] < (W - Wl + 1) * G
+
+
+def test_local_window_zero_is_the_plain_window_and_identical_keys_closed_form():
+    G, W, D, L = 2, 6, 16, 40
+    q, k = rand_bf16((G, W, D), 5), rand_bf16((L, D), 6)
+    a, _, _ = orc.unit_colsum(q, k)
+    b, _, _ = orc.unit_colsum(q, k, local_window=0)
+    assert (a == b).all()
+    # identical keys: a row spreads its weight evenly over the keys it sees
+    Wl = 4
+    kk = k[:1].expand(L, D).contiguous()
+    c, _, _ = orc.unit_colsum(q, kk, local_window=Wl)
+    want = np.zeros(L)
+    for i in range(W):
+        vis = _visible(i, Wl, L)
+        want[:vis] += G / vis
+    np.testing.assert_allclose(c, want, rtol=1e-13)
+
+
+def test_local_window_evict_scores_and_tail():
+    NL, Bt, Hq, Hkv, D, L, W, Wl, kernel, B = 1, 2, 4, 2, 16, 64, 6, 3, 3, 20
+    g = torch.Generator().manual_seed(12)
+    q = bf16(torch.randn((NL, Bt, Hq, W, D), generator=g))
+    k = bf16(torch.randn((NL, Bt, Hkv, L, D), generator=g))
+    v = bf16(torch.randn((NL, Bt, Hkv, L, D), generator=g))
+    R = W
+    out = orc.evict(q, k, v, R, kernel, B, local_window=Wl, want_colsum=True)
+    G = Hq // Hkv
+    for b in range(Bt):
+        for h in range(Hkv):
+            c, _, _ = orc.unit_colsum(q[0, b, h * G:(h + 1) * G], k[0, b, h], local_window=Wl)
+            np.testing.assert_allclose(out["colsum"][0, b, h], c, rtol=1e-14)
+            np.testing.assert_allclose(out["scores"][0, b, h], orc.pool(c, L - R, kernel), rtol=1e-14)
+            assert out["idx"][0, b, h][B - R:].tolist() == list(range(L - R, L))
