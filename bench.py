@@ -48,6 +48,8 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling)")
     ap.add_argument("--prompt-len", type=int, default=0, help="override the prompt length (profiling)")
+    ap.add_argument("--local-window", type=int, default=0,
+                    help="LAQ++ (Eq. 5): this many of the window's queries are causal local queries")
     ap.add_argument("--tiles-per-task", type=int, default=0)
     ap.add_argument("--lag-units", type=int, default=0)
     return ap.parse_args()
@@ -262,6 +264,7 @@ def main():
     idx = torch.empty((NL, Bt, Hkv, B), dtype=torch.int32, device=dev)
     p = laq.params_for(q, k, cfg.keep_tail, cfg.pool_kernel, B, v=v, out=k_out)
     p.tiles_per_task, p.sched_lag_units = args.tiles_per_task, args.lag_units
+    p.local_window = args.local_window
     ws = laq.alloc_workspace(p, dev)
 
     def step():

@@ -12,7 +12,8 @@
  *   Hq, Hkv     query heads, KV heads;  G = Hq / Hkv  query heads share one KV head
  *   D           head dimension (128)
  *   L           prompt length = cached positions before eviction
- *   W           lookahead queries per query head (the observation window)
+ *   W           queries per query head in the observation window: lookahead queries, preceded by
+ *               W_local causal queries of the last prompt positions for LAQ++ (Eq. 5)
  *   R           retained tail: the last R prompt positions are always kept
  *   k           1-D pooling kernel (odd)
  *   B           budget: positions kept per (layer, batch, KV head), tail included
@@ -23,6 +24,8 @@
  * the softmax, the GQA reduction and the pooling, which follow the SnapKV-style "standard KV
  * cache eviction" the paper builds on, Sections 1 and 5.1):
  *   1. logits   s[r][j] = scale * <q_r, k_j>,  r = g*W+i over the G heads x W queries, j in [0,L)
+ *               (a local query i < W_local only sees j <= L - W_local + i; the softmax and the
+ *               column sums below run over the keys a row sees)
  *   2. softmax  P[r][j] = exp(s[r][j]-m_r) / l_r,  m_r = max_j s[r][j],  l_r = sum_j exp(s[r][j]-m_r)
  *   3. column sums  c[j] = sum_r P[r][j]
  *   4. pooling  p[j] = (1/k) * sum_{|t|<=k/2, 0<=j+t<Ls} c[j+t],  j in [0,Ls)   (zero padded)
@@ -91,6 +94,13 @@ typedef struct {
   /* Scheduling knobs of the scoring kernel; 0 lets the library choose. */
   int32_t tiles_per_task;  /* 128-key tiles per scoring task (a task = one sweep over a key chunk) */
   int32_t sched_lag_units; /* how many units the column-sum sweep trails the statistics sweep */
+  /* LAQ++ (Eq. 5, unified window W u Q): the first local_window of each head's window_len queries
+   * are the queries of the last local_window prompt positions (query i at position
+   * L - local_window + i) and attend causally, to positions <= their own; the rest are lookahead
+   * queries and see every prompt key. 0 = plain LAQ (Eq. 4). Needs local_window <= window_len and
+   * local_window <= keep_tail, so that every scored position is visible to every query. */
+  int32_t local_window;
+  int32_t reserved0;       /* must be 0 */
   /* Q [NL][Bt][Hq][W][D] */
   int64_t q_stride_layer, q_stride_batch, q_stride_head, q_stride_pos;
   /* K [NL][Bt][Hkv][L][D] */

@@ -37,7 +37,8 @@ class LaqParams(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "prompt_len", "window_len",
         "keep_tail", "pool_kernel", "pool_mode", "budget")] + [("softmax_scale", ctypes.c_float),
-        ("tiles_per_task", ctypes.c_int32), ("sched_lag_units", ctypes.c_int32)] + [
+        ("tiles_per_task", ctypes.c_int32), ("sched_lag_units", ctypes.c_int32),
+        ("local_window", ctypes.c_int32), ("reserved0", ctypes.c_int32)] + [
         (f"{t}_stride_{d}", ctypes.c_int64) for t in ("q", "k", "v", "o")
         for d in ("layer", "batch", "head", "pos")]
 
@@ -214,7 +215,7 @@ def laq_version() -> int:
 
 def evict(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, budget: int, pool_kernel: int = 7,
           keep_tail: Optional[int] = None, want_scores: bool = False, ws=None, stream=None,
-          softmax_scale: float = 0.0):
+          softmax_scale: float = 0.0, local_window: int = 0):
     """Convenience call: allocates the outputs with torch and runs ``laq_evict``.
 
     q [NL,Bt,Hq,W,D], k and v [NL,Bt,Hkv,L,D], bf16 CUDA tensors. Returns a dict with 'k_out',
@@ -231,6 +232,7 @@ def evict(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, budget: int, pool_k
     scores = torch.empty((NL, Bt, Hkv, L - R), dtype=torch.float32, device=k.device) if want_scores else None
     p = params_for(q, k, R, pool_kernel, budget, v=v, out=k_out)
     p.softmax_scale = softmax_scale  # 0 selects 1/sqrt(head_dim)
+    p.local_window = local_window    # > 0: LAQ++ unified window (Eq. 5)
     if ws is None:
         ws = alloc_workspace(p, k.device)
     laq_evict(p, q, k, v, k_out, v_out, idx, scores, ws, stream)

@@ -21,6 +21,9 @@ laq_status derive_dims(const laq_params* p, Dims* d) {
   if (p->pool_kernel < 1 || (p->pool_kernel % 2) == 0) return LAQ_ERR_INVALID_ARG;
   if (!(p->softmax_scale >= 0.0f) || isinf(p->softmax_scale)) return LAQ_ERR_INVALID_ARG;
   if (p->tiles_per_task < 0 || p->sched_lag_units < 0) return LAQ_ERR_INVALID_ARG;
+  if (p->local_window < 0 || p->local_window > p->window_len || p->local_window > p->keep_tail ||
+      p->reserved0 != 0)
+    return LAQ_ERR_INVALID_ARG;
   if (p->pool_mode != LAQ_POOL_AVG) return LAQ_ERR_UNSUPPORTED;
   if ((p->head_dim % 8) != 0 || p->head_dim > 256) return LAQ_ERR_UNSUPPORTED;
   const int64_t M = (int64_t)(p->n_q_heads / p->n_kv_heads) * p->window_len;
@@ -33,6 +36,7 @@ laq_status derive_dims(const laq_params* p, Dims* d) {
   d->D = p->head_dim;
   d->L = p->prompt_len;
   d->W = p->window_len;
+  d->W_local = p->local_window;
   d->R = p->keep_tail;
   d->kpool = p->pool_kernel;
   d->B = p->budget;

@@ -11,6 +11,7 @@ namespace laq {
 // Problem sizes derived from laq_params (notation of laq.h).
 struct Dims {
   int NL, Bt, Hq, Hkv, G, D, L, W, R, kpool, B;
+  int W_local;  // leading causal queries of each head's window (LAQ++), 0 for plain LAQ
   int M;        // G*W softmax rows per unit
   int Ls, Kb;   // scored positions, selected slots
   int64_t U;    // units

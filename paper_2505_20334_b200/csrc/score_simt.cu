@@ -19,7 +19,7 @@ struct SimtArgs {
   const __nv_bfloat16* k;
   int64_t qs_layer, qs_batch, qs_head, qs_pos;
   int64_t ks_layer, ks_batch, ks_head, ks_pos;
-  int Bt, Hkv, G, W, D, L, M, M_pad, n_part, L_pad, keys_per_chunk;
+  int Bt, Hkv, G, W, W_local, D, L, M, M_pad, n_part, L_pad, keys_per_chunk;
   float scale_log2;  // softmax scale * log2(e)
   float2* part;
   float* row_off;
@@ -80,6 +80,9 @@ __global__ void simt_stats_kernel(SimtArgs a) {
   const int j0 = chunk * a.keys_per_chunk;
   const int j1 = min(a.L, j0 + a.keys_per_chunk);
   const int r = threadIdx.x;
+  // keys this row may see: a causal local query (LAQ++) stops at its own position
+  const int qi = r % a.W;
+  const int vis = qi < a.W_local ? a.L - a.W_local + qi + 1 : a.L;
   float m = -1e30f, l = 0.f;
   for (int js = j0; js < j1; js += kStageKeys) {
     const int nk = min(kStageKeys, j1 - js);
@@ -88,7 +91,7 @@ __global__ void simt_stats_kernel(SimtArgs a) {
       sk[i] = reinterpret_cast<const uint4*>(kbase + (int64_t)(js + i / dv) * a.ks_pos)[i % dv];
     __syncthreads();
     if (r < a.M) {
-      for (int jj = 0; jj < nk; ++jj) {
+      for (int jj = 0; jj < nk && js + jj < vis; ++jj) {
         float acc = 0.f;
         for (int c = 0; c < dv; ++c) acc = dot8(sq[r * qstride4 + c], sk[jj * dv + c], acc);
         const float t = acc * a.scale_log2;
@@ -171,7 +174,7 @@ laq_status score_simt_launch(const laq_params& p, const Dims& d, const Workspace
   a.qs_head = p.q_stride_head;   a.qs_pos = p.q_stride_pos;
   a.ks_layer = p.k_stride_layer; a.ks_batch = p.k_stride_batch;
   a.ks_head = p.k_stride_head;   a.ks_pos = p.k_stride_pos;
-  a.Bt = d.Bt; a.Hkv = d.Hkv; a.G = d.G; a.W = d.W; a.D = d.D; a.L = d.L; a.M = d.M;
+  a.Bt = d.Bt; a.Hkv = d.Hkv; a.G = d.G; a.W = d.W; a.W_local = d.W_local; a.D = d.D; a.L = d.L; a.M = d.M;
   a.M_pad = w.M_pad; a.n_part = w.n_part; a.L_pad = w.L_pad;
   const int n_chunks = w.n_part;
   a.keys_per_chunk = (w.L_pad / TILE_KEYS + n_chunks - 1) / n_chunks * TILE_KEYS;

@@ -58,7 +58,7 @@ constexpr int kTaskConsumers = 4 + kSoftmaxWarps;
 
 struct TcArgs {
   int64_t U;
-  int Bt, Hkv, G, W, L, M, M_pad, n_part, L_pad, n_tiles;
+  int Bt, Hkv, G, W, W_local, L, M, M_pad, n_part, L_pad, n_tiles;
   int tiles_per_task, tasks_per_unit, lag_units;
   uint32_t total_tickets;
   float scale_log2;
@@ -320,18 +320,21 @@ __device__ __forceinline__ void release_buffer(uint32_t empty_bar, int lane) {
   if (lane == 0) mbar_arrive(empty_bar);
 }
 
-// Sweep 1, `valid` (< 64, possibly <= 0) real key columns starting at taddr, out of line: it only
-// occurs in the last tile of a unit whose prompt length is not a multiple of 128.
-__device__ __noinline__ float2 stats_cols_ragged(uint32_t taddr, int valid, float c, float m,
-                                                 float l) {
+// Sweep 1 over up to 64 key columns starting at taddr of which only a part counts, out of line.
+// `valid_max` (warp-uniform, possibly <= 0) bounds the columns that hold real keys; `valid_lane`
+// (<= valid_max) is how many of them this thread's query row may see. It is used for the last tile
+// of a unit whose prompt length is not a multiple of 128 and, with a causal local window (LAQ++,
+// Eq. 5), for the tiles that hold the last prompt positions.
+__device__ __noinline__ float2 stats_cols_ragged(uint32_t taddr, int valid_max, int valid_lane,
+                                                 float c, float m, float l) {
   float v[32];
-  for (int c0 = 0; c0 < valid; c0 += 32) {  // warp-uniform bounds
+  for (int c0 = 0; c0 < valid_max; c0 += 32) {  // warp-uniform bounds
     tmem_ld32(taddr + (uint32_t)c0, v);
     tmem_ld_wait(v);
-    const int nv = valid - c0;
-    float mx = v[0];
+    const int nv = valid_lane - c0;
+    float mx = -3.0e38f;
 #pragma unroll
-    for (int i = 1; i < 32; ++i) mx = (i < nv) ? fmaxf(mx, v[i]) : mx;
+    for (int i = 0; i < 32; ++i) mx = (i < nv) ? fmaxf(mx, v[i]) : mx;
     const float m_new = fmaxf(m, mx * c);
     float sum = 0.f;
 #pragma unroll
@@ -656,6 +659,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
     const int ch_lo = half == 0 ? 0 : (n_chunks2 + 1) / 2;
     const int ch_hi = half == 0 ? (n_chunks2 + 1) / 2 : n_chunks2;
     const uint32_t col0 = 64u * (uint32_t)half;  // sweep 1: this warpgroup's 64 key columns
+    // keys [0, vis) are visible to this thread's query rows: all L for a lookahead query, the
+    // positions up to its own for a local query (query i of a head sits at L - W_local + i)
+    const int qi0 = row_in_wg % a.W, qi1 = (128 + row_in_wg) % a.W;
+    const int vis0 = qi0 < a.W_local ? a.L - a.W_local + qi0 + 1 : a.L;
+    const int vis1 = qi1 < a.W_local ? a.L - a.W_local + qi1 + 1 : a.L;
     // Tiles are numbered through all tasks of this CTA; pair p owns tiles p, p + 2, ... A parity
     // wait is sound because the previous use of a slot (tile t - n_slots) is never later than the
     // pair's previous tile (t - 2).
@@ -693,19 +701,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
           const int valid = min(TILE_KEYS, a.L - key0);
           // row blocks beyond the unit's rows are skipped (warp-uniform)
           const bool rows0 = quad * 32 < a.M, rows1 = RB == 2 && 128 + quad * 32 < a.M;
-          if (valid == TILE_KEYS) {
+          if (valid == TILE_KEYS && key0 + TILE_KEYS <= a.L - a.W_local) {
+            // every column is a real key that every row sees
             if (rows0) stats_cols64(taddr + col0, c, m0, l0, v, !rows1, empty_bar, lane);
             if (rows1) stats_cols64(taddr + 128u + col0, c, m1, l1, v, true, empty_bar, lane);
             if (!rows0) release_buffer(empty_bar, lane);
           } else {
             const int vh = min(64, valid - (int)col0);
             if (rows0) {
-              const float2 r = stats_cols_ragged(taddr + col0, vh, c, m0, l0);
+              const float2 r = stats_cols_ragged(taddr + col0, vh, min(vh, vis0 - key0 - (int)col0), c, m0, l0);
               m0 = r.x;
               l0 = r.y;
             }
             if (rows1) {
-              const float2 r = stats_cols_ragged(taddr + 128u + col0, vh, c, m1, l1);
+              const float2 r =
+                  stats_cols_ragged(taddr + 128u + col0, vh, min(vh, vis1 - key0 - (int)col0), c, m1, l1);
               m1 = r.x;
               l1 = r.y;
             }
@@ -809,7 +819,7 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
                            const void* k, char* ws, cudaStream_t stream, int* launches) {
   TcArgs a;
   a.U = d.U;
-  a.Bt = d.Bt; a.Hkv = d.Hkv; a.G = d.G; a.W = d.W; a.L = d.L; a.M = d.M;
+  a.Bt = d.Bt; a.Hkv = d.Hkv; a.G = d.G; a.W = d.W; a.W_local = d.W_local; a.L = d.L; a.M = d.M;
   a.M_pad = w.M_pad; a.n_part = w.n_part; a.L_pad = w.L_pad;
   a.n_tiles = w.L_pad / TILE_KEYS;
   a.tasks_per_unit = w.n_part;

@@ -28,17 +28,17 @@ def rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed, kscale=1.0):
     return q, k, v
 
 
-def run_evict(laq, q, k, v, R, kernel, B):
+def run_evict(laq, q, k, v, R, kernel, B, local_window=0):
     out = laq.evict(q.cuda(), k.cuda(), v.cuda(), B, pool_kernel=kernel, keep_tail=R,
-                    want_scores=True)
+                    want_scores=True, local_window=local_window)
     assert laq.laq_last_device_status(out["params"], out["ws"]) == laq.LAQ_OK
     return out
 
 
-def compare_all_units(laq, q, k, v, R, kernel, B, out=None):
+def compare_all_units(laq, q, k, v, R, kernel, B, out=None, local_window=0):
     """Full comparison of every unit of a (small) problem against the oracle."""
-    out = out or run_evict(laq, q, k, v, R, kernel, B)
-    ref = orc.evict(q, k, v, R, kernel, B)
+    out = out or run_evict(laq, q, k, v, R, kernel, B, local_window)
+    ref = orc.evict(q, k, v, R, kernel, B, local_window=local_window)
     NL, Bt, Hkv, L = k.shape[0], k.shape[1], k.shape[2], k.shape[3]
     got_scores = out["scores"].cpu().numpy()
     err = score_rel_err(got_scores, ref["scores"])
@@ -195,6 +195,37 @@ def test_evict_identical_keys_ties_go_to_lower_positions(laq):
             assert len(set(got_scores[0, b, h, kernel // 2: Ls - kernel // 2].tolist())) == 1
             assert (idx[0, b, h] == want).all()
             assert (idx[0, b, h] == orc.select(got_scores[0, b, h], L, W, B, sorted_variant=True)).all()
+
+
+LOCAL_SHAPES = [
+    # NL Bt Hq Hkv D    L     W  W_local k  B    what
+    (1, 2, 8, 2, 128, 1028, 16, 8, 7, 120),   # 8 local + 8 lookahead; the window straddles two tiles
+    (1, 1, 4, 1, 128, 777, 32, 16, 7, 200),   # M = 128, ragged last tile
+    (1, 1, 8, 1, 128, 1536, 32, 32, 5, 64),   # M = 256, local queries only (SnapKV-style window)
+    (1, 1, 4, 2, 128, 200, 6, 5, 3, 30),      # window length that is not a power of two
+    (1, 1, 8, 2, 64, 500, 8, 4, 7, 90),       # head_dim 64: CUDA-core path
+]
+
+
+@pytest.mark.parametrize("shape", LOCAL_SHAPES, ids=[f"L{s[5]}-W{s[6]}-local{s[7]}-D{s[4]}" for s in LOCAL_SHAPES])
+def test_unified_window_matches_oracle(laq, shape):
+    NL, Bt, Hq, Hkv, D, L, W, Wl, kernel, B = shape
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=L + Wl, kscale=1.5)
+    err, _ = compare_all_units(laq, q, k, v, W, kernel, B, local_window=Wl)
+    assert err < SCORE_RTOL
+    # the causal mask matters: without it the scores differ
+    plain = run_evict(laq, q, k, v, W, kernel, B)
+    masked = run_evict(laq, q, k, v, W, kernel, B, local_window=Wl)
+    assert not torch.allclose(plain["scores"], masked["scores"], rtol=1e-3, atol=0)
+
+
+def test_local_window_argument_checks(laq):
+    q, k, v = rand_inputs(1, 1, 4, 2, 128, 300, 8, seed=3)
+    for bad in (9, -1):          # longer than the window / negative
+        with pytest.raises(laq.LaqError):
+            laq.evict(q.cuda(), k.cuda(), v.cuda(), 40, keep_tail=8, local_window=bad)
+    with pytest.raises(laq.LaqError):  # local queries must lie inside the retained tail
+        laq.evict(q.cuda(), k.cuda(), v.cuda(), 40, keep_tail=4, local_window=6)
 
 
 def test_extreme_logits_and_late_maximum(laq):
