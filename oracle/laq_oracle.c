@@ -233,3 +233,21 @@ int laq_oracle_evict(const uint16_t* q, const uint16_t* k, const uint16_t* v, in
   return laq_oracle_evict_local(q, k, v, NL, Bt, Hq, Hkv, D, L, W, 0, R, kernel, B, scale, unit_list,
                                 n_units, scores, colsum, idx, k_out, v_out, fast_select);
 }
+
+/*
+ * Recall of a selected index set against a gold one (Section 3, Eq. 1-3):
+ * |M_pred n M_gold| / |M_gold|, by comparing every pair. Both sets hold distinct positions;
+ * no order is assumed. Returns the size of the intersection through *n_common.
+ */
+double laq_oracle_recall(const int32_t* pred, int n_pred, const int32_t* gold, int n_gold,
+                         int32_t* n_common) {
+  int common = 0;
+  for (int a = 0; a < n_pred; ++a)
+    for (int b = 0; b < n_gold; ++b)
+      if (pred[a] == gold[b]) {
+        ++common;
+        break;
+      }
+  if (n_common) *n_common = common;
+  return n_gold > 0 ? (double)common / (double)n_gold : 0.0;
+}

@@ -46,6 +46,8 @@ def _load():
         lib.laq_oracle_evict.argtypes = [vp, vp, vp, i, i, i, i, i, i, i, i, i, i, d, vp, i64,
                                          vp, vp, vp, vp, vp, i]
         lib.laq_oracle_evict.restype = i
+        lib.laq_oracle_recall.argtypes = [vp, i, vp, i, vp]
+        lib.laq_oracle_recall.restype = d
         lib.laq_oracle_evict_local.argtypes = [vp, vp, vp, i, i, i, i, i, i, i, i, i, i, i, d, vp, i64,
                                                vp, vp, vp, vp, vp, i]
         lib.laq_oracle_evict_local.restype = i
@@ -102,6 +104,15 @@ def select(p, L, R, B, sorted_variant=False):
     fn = _load().laq_oracle_select_sorted if sorted_variant else _load().laq_oracle_select
     fn(_ptr(p), L, R, B, _ptr(idx))
     return idx
+
+
+def recall(pred, gold):
+    """(|pred n gold| / |gold|, |pred n gold|) for two sets of distinct positions (Eq. 1-3)."""
+    pred = np.ascontiguousarray(pred, np.int32)
+    gold = np.ascontiguousarray(gold, np.int32)
+    n = np.zeros(1, np.int32)
+    r = _load().laq_oracle_recall(_ptr(pred), pred.shape[0], _ptr(gold), gold.shape[0], _ptr(n))
+    return float(r), int(n[0])
 
 
 def compact(src, idx):

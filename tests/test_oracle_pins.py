@@ -372,3 +372,22 @@ def test_local_window_evict_scores_and_tail():
             np.testing.assert_allclose(out["colsum"][0, b, h], c, rtol=1e-14)
             np.testing.assert_allclose(out["scores"][0, b, h], orc.pool(c, L - R, kernel), rtol=1e-14)
             assert out["idx"][0, b, h][B - R:].tolist() == list(range(L - R, L))
+
+
+# ---------------------------------------------------------------- recall of two index sets (Eq. 1-3)
+def test_recall_hand_cases_and_numpy_intersection():
+    assert orc.recall([1, 2, 3], [4, 5, 6]) == (0.0, 0)
+    assert orc.recall([7, 3, 5], [3, 5, 7]) == (1.0, 3)
+    r, n = orc.recall([0, 2, 4, 6, 8], [1, 2, 3, 4])
+    assert n == 2 and r == pytest.approx(0.5)
+    rng = np.random.default_rng(8)
+    for B, L in ((16, 40), (300, 1000), (64, 64)):
+        a = rng.permutation(L)[:B]
+        b = rng.permutation(L)[:B]
+        r, n = orc.recall(a, b)
+        assert n == len(np.intersect1d(a, b)) and r == pytest.approx(n / B)
+    # selections from the same scores at nested budgets: the smaller set is recalled in full
+    p = rng.random(500)
+    small, big = orc.select(p, 500, 0, 50), orc.select(p, 500, 0, 200)
+    assert orc.recall(big, small) == (1.0, 50)
+    assert orc.recall(small, big)[1] == 50
