@@ -191,6 +191,21 @@ LAQ_API laq_status laq_evict(const laq_params* p, const void* q, const void* k, 
                      size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Recall of one selection against another (Section 3, Eq. 1-3):
+ *     Recall = |M_pred n M_gold| / |M_gold|
+ * per unit, e.g. M_pred from the lookahead window and M_gold from the queries of the real
+ * response, both obtained with laq_score + laq_select.
+ *   idx_pred  device, int32, dense [n_units][n_pred], each row ascending (as laq_select writes it)
+ *   idx_gold  device, int32, dense [n_units][n_gold], each row ascending and without repeats
+ *   n_common  device, int32 [n_units], size of the intersection (may be NULL)
+ *   recall    device, fp32 [n_units] (may be NULL; at least one output is required)
+ * Errors: LAQ_ERR_INVALID_ARG, LAQ_ERR_UNSUPPORTED (more than 2^34 units), LAQ_ERR_CUDA.
+ */
+LAQ_API laq_status laq_recall(int64_t n_units, const int32_t* idx_pred, int32_t n_pred,
+                              const int32_t* idx_gold, int32_t n_gold, int32_t* n_common,
+                              float* recall, void* cuda_stream);
+
+/*
  * The whole step for a cache that lives in HOST memory (ideally pinned): copies Q, K and V to the
  * caller's device staging area, runs laq_evict there and copies the compressed cache back, all
  * ordered on `cuda_stream`. Host tensors are densely packed in the index order of laq_params (the

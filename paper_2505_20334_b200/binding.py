@@ -27,7 +27,7 @@ EXPORTS = (
     "laq_params_dense_strides", "laq_workspace_bytes", "laq_score", "laq_select", "laq_compact",
     "laq_evict", "laq_last_device_status", "laq_last_launch_count", "laq_status_string",
     "laq_version", "laq_set_stage_events", "laq_host_staging_bytes", "laq_evict_host",
-    "laq_score_static",
+    "laq_score_static", "laq_recall",
 )
 
 
@@ -64,6 +64,8 @@ def _load() -> ctypes.CDLL:
     lib.laq_score.restype = ctypes.c_int
     lib.laq_score_static.argtypes = [pp, vp, vp, vp, vp]
     lib.laq_score_static.restype = ctypes.c_int
+    lib.laq_recall.argtypes = [ctypes.c_int64, vp, ctypes.c_int32, vp, ctypes.c_int32, vp, vp, vp]
+    lib.laq_recall.restype = ctypes.c_int
     lib.laq_select.argtypes = [pp, vp, vp, vp]
     lib.laq_select.restype = ctypes.c_int
     lib.laq_compact.argtypes = [pp, vp, vp, vp, vp, vp, vp]
@@ -167,6 +169,24 @@ def laq_score_static(p: LaqParams, q, k, scores, stream=None, check=True) -> int
     if check and st != LAQ_OK:
         raise LaqError(st, "laq_score_static")
     return st
+
+
+def laq_recall(idx_pred: torch.Tensor, idx_gold: torch.Tensor, stream=None):
+    """Recall of `idx_pred` against `idx_gold` (Eq. 1-3) for index tensors [..., B] with ascending
+    rows; returns (recall fp32 [...], n_common int32 [...])."""
+    n_pred, n_gold = idx_pred.shape[-1], idx_gold.shape[-1]
+    lead = idx_pred.shape[:-1]
+    if idx_gold.shape[:-1] != lead:
+        raise ValueError("laq_recall: the two index tensors must agree in all but the last dim")
+    a, g = idx_pred.contiguous(), idx_gold.contiguous()
+    n_units = a.numel() // n_pred
+    common = torch.empty(lead, dtype=torch.int32, device=a.device)
+    rec = torch.empty(lead, dtype=torch.float32, device=a.device)
+    st = lib.laq_recall(n_units, _ptr(a), n_pred, _ptr(g), n_gold, _ptr(common), _ptr(rec),
+                        _stream(stream))
+    if st != LAQ_OK:
+        raise LaqError(st, "laq_recall")
+    return rec, common
 
 
 def laq_select(p: LaqParams, scores, idx, stream=None, check=True) -> int:

@@ -228,6 +228,28 @@ def test_local_window_argument_checks(laq):
         laq.evict(q.cuda(), k.cuda(), v.cuda(), 40, keep_tail=4, local_window=6)
 
 
+def test_recall_of_two_selections_matches_oracle(laq):
+    # Eq. 1-3: the set chosen by a short window against the set chosen by a longer one
+    NL, Bt, Hq, Hkv, D, L, kernel, B = 1, 2, 8, 2, 128, 1500, 7, 128
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, 32, seed=91)
+    gold = run_evict(laq, q, k, v, 8, kernel, B)["idx"]                    # all 32 queries
+    pred = run_evict(laq, q[:, :, :, :8].contiguous(), k, v, 8, kernel, B)["idx"]  # the first 8
+    rec, common = laq.laq_recall(pred, gold)
+    torch.cuda.synchronize()
+    for b in range(Bt):
+        for h in range(Hkv):
+            r, n = orc.recall(pred[0, b, h].cpu().numpy(), gold[0, b, h].cpu().numpy())
+            assert int(common[0, b, h]) == n
+            assert float(rec[0, b, h]) == pytest.approx(r, rel=1e-6)
+            assert 8 <= n < B          # the retained tail is always shared; the rest differs
+    same, n_same = laq.laq_recall(gold, gold)
+    assert (same == 1.0).all() and (n_same == B).all()
+    # different set sizes
+    small = gold[..., :40].contiguous()
+    r2, n2 = laq.laq_recall(small, gold)
+    assert (n2 == 40).all() and torch.allclose(r2, torch.full_like(r2, 40 / B))
+
+
 def test_extreme_logits_and_late_maximum(laq):
     # logits of +-hundreds: the running reference of sweep 1 has to move several times, also in the
     # middle of a task, and sweep 2 sees probabilities far below the smallest fp32 normal
