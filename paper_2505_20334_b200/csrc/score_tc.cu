@@ -14,12 +14,12 @@
 // statistics of every sweep-1 task of the unit; those tasks have smaller tickets, which running
 // CTAs already hold, so the order is deadlock-free for any grid size. Every wait is bounded.
 //
-// Warp roles (672 threads):
+// Warp roles (768 threads):
 //   warp 0       ticket fetch + TMA producer (one lane)
 //   warps 1, 20  tcgen05.mma issuers for alternate tiles (one lane each); warp 1 owns the TMEM
 //   warp 2       statistics out: merges the warpgroups' (shift, sum) of a finished sweep-1 task,
 //                writes the task's partial to global memory and bumps the unit's counter
-//   warp 3       statistics in: for a sweep-2 task, waits for the unit's counter, merges the
+//   warps 3, 21-23  statistics in: for a sweep-2 task, wait for the unit's counter, merge the
 //                unit's partials into -b_r and hands them to the softmax warps in shared memory
 //   warps 4-19   four softmax warpgroups in two pairs. Pair p takes the tiles t with t mod 2 == p;
 //                inside a pair the two warpgroups split the accumulator's columns in half, so a
@@ -45,7 +45,8 @@ using namespace laq::math;
 constexpr int kSoftmaxWgs = 4;
 constexpr int kSoftmaxWarps = 4 * kSoftmaxWgs;
 constexpr int kMmaWarpB = 4 + kSoftmaxWarps;  // index of the second MMA issuer's warp
-constexpr int kThreads = 32 * (kMmaWarpB + 1);
+constexpr int kStatInWarps = 4;               // warp 3 and the warps after the second MMA issuer
+constexpr int kThreads = 32 * (kMmaWarpB + kStatInWarps);
 constexpr int kTaskSlots = 4;
 constexpr int kMaxSlots = 4;  // K stages in shared memory = TMEM accumulator buffers
 constexpr int kStatSlots = 2;
@@ -53,8 +54,8 @@ constexpr uint32_t kKStageBytes = TILE_KEYS * 128 * 2;  // 128 keys x 128 dims x
 constexpr uint32_t kCtlBytes = 22528;
 constexpr long long kTimeoutCycles = 4000000000LL;  // ~2 s: every device-side wait gives up after this
 constexpr float kLog2e = 1.4426950408889634f;
-// two MMA lanes, statistics-out warp, statistics-in warp, softmax warps
-constexpr int kTaskConsumers = 4 + kSoftmaxWarps;
+// two MMA lanes, statistics-out warp, statistics-in warps, softmax warps
+constexpr int kTaskConsumers = 3 + kStatInWarps + kSoftmaxWarps;
 
 struct TcArgs {
   int64_t U;
@@ -395,7 +396,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
     for (int i = 0; i < kStatSlots; ++i) {
       mbar_init(smem_u32(&ctl->stat_full[i]), kSoftmaxWarps);
       mbar_init(smem_u32(&ctl->stat_empty[i]), 1);
-      mbar_init(smem_u32(&ctl->boff_full[i]), 1);
+      mbar_init(smem_u32(&ctl->boff_full[i]), kStatInWarps);
       mbar_init(smem_u32(&ctl->boff_empty[i]), kSoftmaxWarps);
     }
     ctl->abort = 0;
@@ -593,8 +594,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       }
       ++sc;
     }
-  } else if (warp == 3) {
+  } else if (warp == 3 || warp > kMmaWarpB) {
     // ================= statistics in =================
+    // four warps, one thread per softmax row (two for 256 rows)
+    const int sin_tid = (warp == 3 ? 0 : warp - kMmaWarpB) * 32 + lane;  // 0..127
     uint32_t tk = 0, sc = 0;
     while (true) {
       Task task;
@@ -622,18 +625,25 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       ready = __shfl_sync(0xffffffffu, ready, 0);
       if (!ready) break;
       const float2* src = a.part + (int64_t)task.unit * a.n_part * a.M_pad;
-      for (int row = lane; row < 256; row += 32) {
+      for (int row = sin_tid; row < 256; row += 32 * kStatInWarps) {
         float nb = -1e30f;
         if (row < a.M) {
           float m = -1e30f, l = 0.f;
           const float2* pp = src + row;
           int c0 = 0;
-          for (; c0 + 16 <= a.tasks_per_unit; c0 += 16) {
-            float2 pr[16];
+          for (; c0 + 32 <= a.tasks_per_unit; c0 += 32) {
+            float2 pr[32];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) pr[i] = __ldcg(pp + (int64_t)(c0 + i) * a.M_pad);
+            for (int i = 0; i < 32; ++i) pr[i] = __ldcg(pp + (int64_t)(c0 + i) * a.M_pad);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) merge_stat(m, l, pr[i]);
+            for (int i = 0; i < 32; ++i) merge_stat(m, l, pr[i]);
+          }
+          for (; c0 + 8 <= a.tasks_per_unit; c0 += 8) {
+            float2 pr[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pr[i] = __ldcg(pp + (int64_t)(c0 + i) * a.M_pad);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) merge_stat(m, l, pr[i]);
           }
           for (; c0 < a.tasks_per_unit; ++c0) merge_stat(m, l, __ldcg(pp + (int64_t)c0 * a.M_pad));
           nb = -(m + log2f(l));
@@ -834,11 +844,18 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
     return LAQ_ERR_CUDA;
-  // sweep 2 trails sweep 1 by enough tasks that the statistics it needs are normally final
+  // Sweep 2 trails sweep 1 by `lag` units. Too short and sweep-2 tasks wait for statistics that
+  // are not final yet; too long and K has left L2 when the second sweep reads it again. Measured
+  // on B200 (8 MiB of K per unit): 48 MiB of K between the sweeps re-reads everything from L2
+  // (9.3 GB of DRAM traffic per 8.6 GB of K), 64 MiB re-reads everything from HBM (15.8 GB); and
+  // about 1.3 tickets per SM is the shortest distance at which sweep 2 rarely waits.
   int lag = d.sched_lag_units;
-  // (measured on B200: about 1.6 tickets per SM between the two sweeps of a unit is the smallest
-  // distance at which sweep-2 tasks rarely wait; a larger one only pushes K further out of L2)
-  if (lag <= 0) lag = (13 * sms / 8 + 2 * a.tasks_per_unit - 1) / (2 * a.tasks_per_unit);
+  if (lag <= 0) {
+    const int64_t k_unit_bytes = (int64_t)d.L * d.D * 2;
+    const int by_l2 = (int)((48ll << 20) / (k_unit_bytes > 0 ? k_unit_bytes : 1));
+    const int by_latency = (5 * sms / 4 + 2 * a.tasks_per_unit - 1) / (2 * a.tasks_per_unit);
+    lag = by_l2 > by_latency ? by_l2 : by_latency;
+  }
   if ((int64_t)lag > d.U) lag = (int)d.U;
   a.lag_units = lag;
   a.scale_log2 = d.scale * kLog2e;

@@ -10,11 +10,12 @@
 #ifndef LAQ_POLY_PAIRS_S1
 // Of every 8 element pairs, how many take the FMA-pipe exp2 instead of the MUFU. Alone, the
 // arithmetic is fastest at 2-3 of 8 (MUFU-bound below, FMA-bound above); inside the kernel on a
-// power-capped B200 0, 2 and 4 of 8 time within 1 % of each other.
-#define LAQ_POLY_PAIRS_S1 2
+// B200 at its power cap the MUFU is the cheaper unit: 0 of 8 is 2 % faster than 2 of 8 and 6 %
+// faster than 4 of 8 (the GPU parity suite passes with 2 of 8 as well).
+#define LAQ_POLY_PAIRS_S1 0
 #endif
 #ifndef LAQ_POLY_PAIRS_S2
-#define LAQ_POLY_PAIRS_S2 2  // same for sweep 2 (even)
+#define LAQ_POLY_PAIRS_S2 0  // same for sweep 2 (even)
 #endif
 
 namespace laq {
