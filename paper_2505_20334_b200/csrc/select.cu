@@ -166,14 +166,37 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const float* _
 }
 
 // Steps 4 and 5 for units of at most kRegItems * 1024 scored positions, with the unit's pooled
-// scores held in registers (kRegItems per thread) instead of memory. Warp w owns the contiguous
-// positions [1024 w, 1024 w + 1024), lane-strided, which is also the order the kept positions are
-// written in. The key of the Kb-th largest score is built bit by bit from the top: a candidate
-// bit stays set if at least Kb keys are >= the candidate; each step is 32 register compares per
-// thread, one warp reduction and one block barrier, with no atomics and no memory passes.
+// scores held in registers (kRegItems = 32 per thread) instead of memory. Warp w owns the
+// contiguous positions [1024 w, 1024 w + 1024), lane-strided, which is also the order the kept
+// positions are written in.
+// The key of the Kb-th largest score is found bit by bit from the top, on bit planes: each thread
+// transposes its 32 keys into 32 words (word b holds bit b of every key), so that one step is an
+// AND and a population count per thread plus one block-wide sum -- no atomics, no memory passes.
+// `alive` marks the keys that agree with the threshold's bits so far; if the alive keys with the
+// current bit set, together with the keys already known to lie above, reach Kb, the bit is 1 and
+// only those stay alive; otherwise the bit is 0 and they join the keys above.
 // The pooling arithmetic is that of pool_kernel, so the scores are bit-identical to laq_score's.
 constexpr int kRegItems = 32;
 
+// In-register transpose of a 32 x 32 bit matrix: on return bit i of a[b] is bit b of the old a[i].
+__device__ __forceinline__ void transpose32(uint32_t (&a)[32]) {
+  uint32_t m = 0x0000ffffu;
+#pragma unroll
+  for (int j = 16; j != 0; j >>= 1, m ^= m << j) {
+#pragma unroll
+    for (int k = 0; k < 32; ++k) {
+      if ((k & j) == 0) {
+        // swap the high-j block of row k with the low-j block of row k + j
+        const uint32_t t = ((a[k] >> j) ^ a[k + j]) & m;
+        a[k + j] ^= t;
+        a[k] ^= t << j;
+      }
+    }
+  }
+}
+
+// kPoolStatic > 0 fixes the pooling kernel at compile time (unrolled taps); 0 takes it from `kpool`.
+template <int kPoolStatic>
 __global__ void __launch_bounds__(kSelThreads) pool_select_reg_kernel(
     const float* __restrict__ colsum, int L_pad, float* pooled_out, int32_t* __restrict__ idx, int Ls,
     int Kb, int R, int B, int kpool, float inv_k) {
@@ -184,70 +207,80 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_reg_kernel(
   int32_t* out = idx + u * (int64_t)B;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int base = warp * (kRegItems * 32) + lane;
-  const int h = kpool / 2;
+  const int h = (kPoolStatic > 0 ? kPoolStatic : kpool) / 2;
 
-  uint32_t keys[kRegItems];
+  uint32_t w[kRegItems];  // first the keys, then their bit planes
+  uint32_t alive = 0u;    // bit `it` set: item `it` of this thread is a real position
 #pragma unroll
   for (int it = 0; it < kRegItems; ++it) {
     const int j = base + it * 32;
-    uint32_t key = 0u;  // below the key of every real score
+    uint32_t key = 0u;
     if (j < Ls) {
       float acc = 0.f;
-      for (int t = -h; t <= h; ++t) {
-        const int jj = j + t;
-        if (jj >= 0 && jj < Ls) acc += c[jj];
+      if (j >= h && j + h < Ls) {
+        if (kPoolStatic > 0) {
+#pragma unroll
+          for (int t = -(kPoolStatic / 2); t <= kPoolStatic / 2; ++t) acc += c[j + t];
+        } else {
+          for (int t = -h; t <= h; ++t) acc += c[j + t];
+        }
+      } else {
+        for (int t = -h; t <= h; ++t) {
+          const int jj = j + t;
+          if (jj >= 0 && jj < Ls) acc += c[jj];
+        }
       }
       const float pj = acc * inv_k;
       if (pooled_out) pooled_out[u * (int64_t)Ls + j] = pj;
       key = order_key(pj);
+      alive |= 1u << it;
     }
-    keys[it] = key;
+    w[it] = key;
   }
+  // w[i] bit b = bit b of key i  ->  w[b] bit i = bit b of key i
+  transpose32(w);
 
-  // number of keys >= cand in the whole block (every warp computes the total)
-  int step = 0;
-  auto count_ge = [&](uint32_t cand) -> uint32_t {
-    uint32_t n = 0;
-#pragma unroll
-    for (int it = 0; it < kRegItems; ++it) n += keys[it] >= cand ? 1u : 0u;
-    n = __reduce_add_sync(0xffffffffu, n);
-    uint32_t* slot = s_cnt[step & 1];
-    ++step;
-    if (lane == 0) slot[warp] = n;
-    __syncthreads();
-    return __reduce_add_sync(0xffffffffu, slot[lane]);
-  };
+  uint32_t above_mask = 0u;  // items known to lie above the threshold
+  uint32_t above = 0u;       // their number in the whole block
   uint32_t theta = 0u;
-#pragma unroll 1
-  for (int bit = 31; bit >= 0; --bit) {
-    const uint32_t cand = theta | (1u << bit);
-    if (count_ge(cand) >= (uint32_t)Kb) theta = cand;
-  }
-  // theta is the key of the Kb-th largest score; `need` positions holding exactly theta are kept
-  const uint32_t n_above = theta == 0xffffffffu ? 0u : count_ge(theta + 1u);
-  const uint32_t need = (uint32_t)Kb - n_above;
-
-  uint32_t n_gt = 0, n_eq = 0;
 #pragma unroll
-  for (int it = 0; it < kRegItems; ++it) {
-    n_gt += __popc(__ballot_sync(0xffffffffu, keys[it] > theta));
-    n_eq += __popc(__ballot_sync(0xffffffffu, keys[it] == theta));
+  for (int bit = 31; bit >= 0; --bit) {
+    const uint32_t ones = w[bit] & alive;
+    const uint32_t n_warp = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(ones));
+    uint32_t* slot = s_cnt[bit & 1];
+    if (lane == 0) slot[warp] = n_warp;
+    __syncthreads();
+    const uint32_t n = __reduce_add_sync(0xffffffffu, slot[lane]);
+    if (above + n >= (uint32_t)Kb) {
+      theta |= 1u << bit;
+      alive = ones;
+    } else {
+      above += n;
+      above_mask |= ones;
+      alive ^= ones;
+    }
   }
+  // `alive` now marks the items whose key equals theta, the key of the Kb-th largest score;
+  // `need` of them are kept (the lowest positions first), with all `above` items
+  const uint32_t need = (uint32_t)Kb - above;
+
+  const uint32_t n_gt = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(above_mask));
+  const uint32_t n_eq = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(alive));
   if (lane == 0) {
     s_gt[warp] = n_gt;
     s_eq[warp] = n_eq;
   }
   __syncthreads();
   uint32_t gt_run = 0, eq_run = 0;
-  for (int w = 0; w < warp; ++w) {
-    gt_run += s_gt[w];
-    eq_run += s_eq[w];
+  for (int ww = 0; ww < warp; ++ww) {
+    gt_run += s_gt[ww];
+    eq_run += s_eq[ww];
   }
   const uint32_t lt_mask = (1u << lane) - 1u;
 #pragma unroll
   for (int it = 0; it < kRegItems; ++it) {
-    const bool gt = keys[it] > theta;
-    const bool eq = keys[it] == theta;
+    const bool gt = (above_mask >> it) & 1u;
+    const bool eq = (alive >> it) & 1u;
     const uint32_t bg = __ballot_sync(0xffffffffu, gt);
     const uint32_t be = __ballot_sync(0xffffffffu, eq);
     const uint32_t gt_before = gt_run + __popc(bg & lt_mask);
@@ -292,8 +325,19 @@ laq_status pool_select_launch(const Dims& d, const float* colsum, int L_pad, flo
   *done = false;
   if (d.U > 0x7fffffff) return LAQ_OK;
   if (d.Ls <= kRegItems * kSelThreads) {
-    pool_select_reg_kernel<<<(unsigned)d.U, kSelThreads, 0, stream>>>(
-        colsum, L_pad, pooled_out, idx, d.Ls, d.Kb, d.R, d.B, d.kpool, 1.0f / (float)d.kpool);
+    const float inv_k = 1.0f / (float)d.kpool;
+    const unsigned grid = (unsigned)d.U;
+#define LAQ_LAUNCH_POOL_SELECT(KP)                                                         \
+  pool_select_reg_kernel<KP><<<grid, kSelThreads, 0, stream>>>(colsum, L_pad, pooled_out, idx, \
+                                                               d.Ls, d.Kb, d.R, d.B, d.kpool, inv_k)
+    switch (d.kpool) {
+      case 1: LAQ_LAUNCH_POOL_SELECT(1); break;
+      case 3: LAQ_LAUNCH_POOL_SELECT(3); break;
+      case 5: LAQ_LAUNCH_POOL_SELECT(5); break;
+      case 7: LAQ_LAUNCH_POOL_SELECT(7); break;
+      default: LAQ_LAUNCH_POOL_SELECT(0); break;
+    }
+#undef LAQ_LAUNCH_POOL_SELECT
     *launches += 1;
     *done = true;
     return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;
