@@ -315,6 +315,14 @@ def main():
                 "unit": "GB/s", "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES,
                 "peak_source": peak_src, "algorithmic_bytes_per_launch": score_bytes,
                 "kernel_ms": score_ms, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
+    # The scoring kernel's busiest unit is the MUFU: two base-2 exponentials per (row, key) pair
+    # (one per sweep) at 16 per clock and SM.
+    n_exp = 2.0 * cfg.units * cfg.rows * cfg.prompt_len
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    mufu_peak = 16.0 * sms * (clocks.get("sm_max_mhz") or 1965) * 1e6
+    roofline["mufu"] = {"bound": "alu", "achieved": n_exp / (score_ms * 1e-3), "peak": mufu_peak,
+                        "unit": "ex2/s", "frac": n_exp / (score_ms * 1e-3) / mufu_peak,
+                        "peak_source": "16 ex2 per clock and SM (measured) x SMs x max SM clock"}
     step_gbs = (score_bytes + gather_bytes) / (ms_per_step * 1e-3) / 1e9
     step_roofline = {"algorithmic_bytes_per_step": score_bytes + gather_bytes, "achieved": step_gbs,
                      "unit": "GB/s", "frac_of_measured": step_gbs / peak,
