@@ -263,6 +263,29 @@ def evict(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, budget: int, pool_k
 
 
 
+def evict_layer_budgets(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, budgets, pool_kernel: int = 7,
+                        keep_tail: Optional[int] = None, local_window: int = 0, stream=None):
+    """Eviction with one budget per layer (the paper fixes the budget, Section 5.2, and names
+    layer-wise budgets such as PyramidKV's as a combination). The units of different layers are
+    independent, so this is one ``laq_evict`` call per run of layers that share a budget, on layer
+    slices of the same tensors (no copies). Returns a list with one dict per layer
+    ('k_out', 'v_out' [Bt,Hkv,B_l,D], 'idx' [Bt,Hkv,B_l])."""
+    NL = q.shape[0]
+    if len(budgets) != NL:
+        raise ValueError("evict_layer_budgets: one budget per layer is required")
+    out, ws, lo = [None] * NL, None, 0
+    while lo < NL:
+        hi = lo + 1
+        while hi < NL and budgets[hi] == budgets[lo]:
+            hi += 1
+        r = evict(q[lo:hi], k[lo:hi], v[lo:hi], int(budgets[lo]), pool_kernel=pool_kernel,
+                  keep_tail=keep_tail, stream=stream, local_window=local_window)
+        for n in range(lo, hi):
+            out[n] = {"k_out": r["k_out"][n - lo], "v_out": r["v_out"][n - lo], "idx": r["idx"][n - lo]}
+        lo = hi
+    return out
+
+
 def laq_host_staging_bytes(p: LaqParams) -> int:
     return int(lib.laq_host_staging_bytes(ctypes.byref(p)))
 

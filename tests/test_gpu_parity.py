@@ -250,6 +250,23 @@ def test_recall_of_two_selections_matches_oracle(laq):
     assert (n2 == 40).all() and torch.allclose(r2, torch.full_like(r2, 40 / B))
 
 
+def test_layer_wise_budgets_on_layer_slices(laq):
+    # a pyramid of budgets: each run of equal budgets is one call on a slice of the layer dimension
+    NL, Bt, Hq, Hkv, D, L, W, kernel = 4, 1, 4, 2, 128, 640, 8, 7
+    budgets = [96, 96, 48, 24]
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=61)
+    outs = laq.evict_layer_budgets(q.cuda(), k.cuda(), v.cuda(), budgets, pool_kernel=kernel)
+    torch.cuda.synchronize()
+    for n, B in enumerate(budgets):
+        ref = orc.evict(q[n:n + 1], k[n:n + 1], v[n:n + 1], W, kernel, B)
+        got = outs[n]["idx"].cpu().numpy()
+        for b in range(Bt):
+            for h in range(Hkv):
+                check_index_set(got[b, h], ref["idx"][0, b, h], ref["scores"][0, b, h], L, W, B)
+                assert (bits(outs[n]["k_out"][b, h]) == bits(k[n, b, h])[got[b, h]]).all()
+                assert (bits(outs[n]["v_out"][b, h]) == bits(v[n, b, h])[got[b, h]]).all()
+
+
 def test_extreme_logits_and_late_maximum(laq):
     # logits of +-hundreds: the running reference of sweep 1 has to move several times, also in the
     # middle of a task, and sweep 2 sees probabilities far below the smallest fp32 normal
