@@ -70,7 +70,7 @@ class ClockSampler(threading.Thread):
     def __init__(self, device_index: int, period_s: float = 0.01):
         super().__init__(daemon=True)
         self.period = period_s
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.power_w, self.reasons, self.max_mhz = [], [], set(), None
         self._stop_evt = threading.Event()
         self.handle = None
         try:
@@ -105,6 +105,10 @@ class ClockSampler(threading.Thread):
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM))
                 try:
+                    self.power_w.append(nv.nvmlDeviceGetPowerUsage(self.handle) / 1000.0)
+                except Exception:
+                    pass
+                try:
                     r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
                 except Exception:
                     r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle)
@@ -122,7 +126,9 @@ class ClockSampler(threading.Thread):
         if self.samples:
             s = sorted(self.samples)
             med = s[len(s) // 2]
-        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+        return {"sm_mhz": med, "sm_min_mhz": min(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "power_w_max": max(self.power_w) if self.power_w else None,
                 "samples": len(self.samples)}
 
 

@@ -108,6 +108,43 @@ void laq_oracle_pool(const double* c, int Ls, int kernel, double* p) {
 }
 
 /*
+ * Step 4 with maximum pooling instead (the other pooling the SnapKV-style step is used with):
+ * p_j = max of c over the window positions that exist, |t| <= k/2 and 0 <= j+t < Ls. Positions
+ * outside [0, Ls) are not candidates (padding with minus infinity).
+ */
+void laq_oracle_pool_max(const double* c, int Ls, int kernel, double* p) {
+  const int h = kernel / 2;
+  for (int j = 0; j < Ls; ++j) {
+    double best = c[j];
+    for (int t = -h; t <= h; ++t) {
+      const int jj = j + t;
+      if (jj >= 0 && jj < Ls && c[jj] > best) best = c[jj];
+    }
+    p[j] = best;
+  }
+}
+
+/*
+ * Eq. 4 read literally: the importance of key j is the sum of the raw (scaled) logits
+ * "sum_{q_i in Q} q_i K^T" over the window rows, with no softmax. Same arguments as
+ * laq_oracle_unit_colsum; c[j] may be negative.
+ */
+void laq_oracle_unit_rawsum(const uint16_t* q, const uint16_t* k, int G, int W, int D, int L,
+                            double scale, double* c) {
+  const int M = G * W;
+  for (int j = 0; j < L; ++j) {
+    double total = 0.0;
+    for (int r = 0; r < M; ++r) {
+      double acc = 0.0;
+      for (int d = 0; d < D; ++d)
+        acc += bf16_to_double(q[(size_t)r * D + d]) * bf16_to_double(k[(size_t)j * D + d]);
+      total += scale * acc;
+    }
+    c[j] = total;
+  }
+}
+
+/*
  * Step 5 (Eq. 4's ArgSort(...)[:B], descending): the Kb = B-R positions of largest p, a tie
  * going to the lower position; written ascending and followed by the tail Ls..L-1.
  * Selection by repeated scan for the best remaining position: O(Ls*Kb), obviously correct.
@@ -180,13 +217,45 @@ void laq_oracle_compact(const uint16_t* src, const int32_t* idx, int B, int D, u
  * u = (layer*Bt + b)*Hkv + h; outputs of other units are left untouched.
  * Query head h*G+g belongs to KV head h. Returns the number of OpenMP threads used.
  */
+/*
+ * Variants of the step (all off when the structure is zeroed):
+ *   W_local    unified window of LAQ++ (Eq. 5), see laq_oracle_unit_colsum_local
+ *   pool_mode  0 average pooling, 1 maximum pooling
+ *   score_mode 0 attention weights (softmax), 1 raw logit sums (Eq. 4 read literally)
+ *   seq_lens   [Bt] or NULL: prompt b holds only its first seq_lens[b] <= L positions. Everything
+ *              is then taken relative to that length Lb: keys [0, Lb), local queries at the last
+ *              W_local of them, scored positions [0, Lb-R), tail [Lb-R, Lb). Scores and column
+ *              sums beyond are written as 0; rows of K/V beyond Lb are never read.
+ */
+typedef struct {
+  int32_t W_local, pool_mode, score_mode, reserved;
+  const int32_t* seq_lens;
+} laq_oracle_variant;
+
+int laq_oracle_evict_variant(const uint16_t* q, const uint16_t* k, const uint16_t* v, int NL, int Bt,
+                             int Hq, int Hkv, int D, int L, int W, int R, int kernel, int B,
+                             double scale, const laq_oracle_variant* var, const int64_t* unit_list,
+                             int64_t n_units, double* scores, double* colsum, int32_t* idx,
+                             uint16_t* k_out, uint16_t* v_out, int fast_select);
+
 int laq_oracle_evict_local(const uint16_t* q, const uint16_t* k, const uint16_t* v, int NL, int Bt,
                            int Hq, int Hkv, int D, int L, int W, int W_local, int R, int kernel, int B,
-                     double scale, const int64_t* unit_list, int64_t n_units, double* scores,
-                     double* colsum, int32_t* idx, uint16_t* k_out, uint16_t* v_out,
-                     int fast_select) {
+                           double scale, const int64_t* unit_list, int64_t n_units, double* scores,
+                           double* colsum, int32_t* idx, uint16_t* k_out, uint16_t* v_out,
+                           int fast_select) {
+  laq_oracle_variant var;
+  memset(&var, 0, sizeof var);
+  var.W_local = W_local;
+  return laq_oracle_evict_variant(q, k, v, NL, Bt, Hq, Hkv, D, L, W, R, kernel, B, scale, &var,
+                                  unit_list, n_units, scores, colsum, idx, k_out, v_out, fast_select);
+}
+
+int laq_oracle_evict_variant(const uint16_t* q, const uint16_t* k, const uint16_t* v, int NL, int Bt,
+                             int Hq, int Hkv, int D, int L, int W, int R, int kernel, int B,
+                             double scale, const laq_oracle_variant* var, const int64_t* unit_list,
+                             int64_t n_units, double* scores, double* colsum, int32_t* idx,
+                             uint16_t* k_out, uint16_t* v_out, int fast_select) {
   const int G = Hq / Hkv;
-  const int Ls = L - R;
   const int64_t U = (int64_t)NL * Bt * Hkv;
   const int64_t n = unit_list ? n_units : U;
   int threads = 1;
@@ -204,18 +273,27 @@ int laq_oracle_evict_local(const uint16_t* q, const uint16_t* k, const uint16_t*
     const int64_t lb = u / Hkv; /* layer*Bt + b */
     const uint16_t* qu = q + ((lb * Hq + h * G) * (int64_t)W) * D;
     const uint16_t* ku = k + u * (int64_t)L * D;
-    double* c = (double*)malloc((size_t)L * sizeof(double));
-    double* p = (double*)malloc((size_t)(Ls > 0 ? Ls : 1) * sizeof(double));
-    laq_oracle_unit_colsum_local(qu, ku, G, W, W_local, D, L, scale, c, NULL, NULL);
-    laq_oracle_pool(c, Ls, kernel, p);
+    /* this prompt's own length, and the scored positions that follow from it */
+    const int Lb = var->seq_lens ? var->seq_lens[lb % Bt] : L;
+    const int Ls = Lb - R;
+    double* c = (double*)calloc((size_t)L, sizeof(double));
+    double* p = (double*)calloc((size_t)(L - R > 0 ? L - R : 1), sizeof(double));
+    if (var->score_mode == 1)
+      laq_oracle_unit_rawsum(qu, ku, G, W, D, Lb, scale, c);
+    else
+      laq_oracle_unit_colsum_local(qu, ku, G, W, var->W_local, D, Lb, scale, c, NULL, NULL);
+    if (var->pool_mode == 1)
+      laq_oracle_pool_max(c, Ls, kernel, p);
+    else
+      laq_oracle_pool(c, Ls, kernel, p);
     if (colsum) memcpy(colsum + u * (int64_t)L, c, (size_t)L * sizeof(double));
-    if (scores) memcpy(scores + u * (int64_t)Ls, p, (size_t)Ls * sizeof(double));
+    if (scores) memcpy(scores + u * (int64_t)(L - R), p, (size_t)(L - R) * sizeof(double));
     if (idx) {
       int32_t* iu = idx + u * (int64_t)B;
       if (fast_select)
-        laq_oracle_select_sorted(p, L, R, B, iu);
+        laq_oracle_select_sorted(p, Lb, R, B, iu);
       else
-        laq_oracle_select(p, L, R, B, iu);
+        laq_oracle_select(p, Lb, R, B, iu);
       if (k_out) laq_oracle_compact(ku, iu, B, D, k_out + u * (int64_t)B * D);
       if (v_out) laq_oracle_compact(v + u * (int64_t)L * D, iu, B, D, v_out + u * (int64_t)B * D);
     }

@@ -26,6 +26,12 @@ def build(force: bool = False) -> str:
     return _LIB
 
 
+class _Variant(ctypes.Structure):
+    _fields_ = [("W_local", ctypes.c_int32), ("pool_mode", ctypes.c_int32),
+                ("score_mode", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("seq_lens", ctypes.c_void_p)]
+
+
 def _load():
     global _lib
     if _lib is None:
@@ -51,6 +57,14 @@ def _load():
         lib.laq_oracle_evict_local.argtypes = [vp, vp, vp, i, i, i, i, i, i, i, i, i, i, i, d, vp, i64,
                                                vp, vp, vp, vp, vp, i]
         lib.laq_oracle_evict_local.restype = i
+        lib.laq_oracle_pool_max.argtypes = [vp, i, i, vp]
+        lib.laq_oracle_pool_max.restype = None
+        lib.laq_oracle_unit_rawsum.argtypes = [vp, vp, i, i, i, i, d, vp]
+        lib.laq_oracle_unit_rawsum.restype = None
+        lib.laq_oracle_evict_variant.argtypes = [vp, vp, vp, i, i, i, i, i, i, i, i, i, i, d,
+                                                 ctypes.POINTER(_Variant), vp, i64,
+                                                 vp, vp, vp, vp, vp, i]
+        lib.laq_oracle_evict_variant.restype = i
         _lib = lib
     return _lib
 
@@ -88,12 +102,25 @@ def unit_colsum(q, k, scale=None, local_window=0):
     return c, m, l
 
 
-def pool(c, Ls, kernel):
+def pool(c, Ls, kernel, mode=0):
+    """mode 0: average pooling (zero padding, divisor k); mode 1: maximum pooling."""
     c = np.ascontiguousarray(c, np.float64)
     assert c.shape[0] >= Ls
     p = np.empty(Ls, np.float64)
-    _load().laq_oracle_pool(_ptr(c), Ls, kernel, _ptr(p))
+    fn = _load().laq_oracle_pool_max if mode == 1 else _load().laq_oracle_pool
+    fn(_ptr(c), Ls, kernel, _ptr(p))
     return p
+
+
+def unit_rawsum(q, k, scale=None):
+    """q [G][W][D], k [L][D] (bf16) -> c [L]: sums of the raw scaled logits over the window rows."""
+    q, k = _bits(q), _bits(k)
+    G, W, D = q.shape
+    L = k.shape[0]
+    scale = 1.0 / np.sqrt(D) if scale is None else float(scale)
+    c = np.empty(L, np.float64)
+    _load().laq_oracle_unit_rawsum(_ptr(q), _ptr(k), G, W, D, L, scale, _ptr(c))
+    return c
 
 
 def select(p, L, R, B, sorted_variant=False):
@@ -124,12 +151,14 @@ def compact(src, idx):
 
 
 def evict(q, k, v, R, kernel, B, scale=None, units=None, want_colsum=False, fast_select=True,
-          want_idx=True, local_window=0):
+          want_idx=True, local_window=0, pool_mode=0, score_mode=0, seq_lens=None):
     """Whole step on dense tensors. q [NL][Bt][Hq][W][D], k/v [NL][Bt][Hkv][L][D] (bf16).
 
     Returns a dict with 'scores' [NL,Bt,Hkv,L-R] fp64, 'idx' [NL,Bt,Hkv,B] int32, 'k_out',
     'v_out' [NL,Bt,Hkv,B,D] uint16 bit patterns, 'threads', and 'colsum' if asked. With `units`
     (unit numbers (layer*Bt+b)*Hkv+h) only those units are computed; the rest stays zero.
+    `pool_mode` 1 pools by maximum, `score_mode` 1 sums raw logits instead of attention weights,
+    `seq_lens` [Bt] gives every prompt its own length (<= L).
     """
     q, k = _bits(q), _bits(k)
     v = None if v is None else _bits(v)
@@ -144,9 +173,12 @@ def evict(q, k, v, R, kernel, B, scale=None, units=None, want_colsum=False, fast
     k_out = np.zeros((NL, Bt, Hkv, B, D), np.uint16) if want_idx else None
     v_out = np.zeros((NL, Bt, Hkv, B, D), np.uint16) if (want_idx and v is not None) else None
     ul = None if units is None else np.ascontiguousarray(units, np.int64)
-    threads = _load().laq_oracle_evict_local(
-        _ptr(q), _ptr(k), _ptr(v), NL, Bt, Hq, Hkv, D, L, W, int(local_window), R, kernel, B, scale, _ptr(ul),
-        0 if ul is None else ul.shape[0], _ptr(scores), _ptr(colsum), _ptr(idx), _ptr(k_out),
+    sl = None if seq_lens is None else np.ascontiguousarray(seq_lens, np.int32)
+    assert sl is None or (sl.shape == (Bt,) and (sl <= L).all() and (sl > B).all())
+    var = _Variant(int(local_window), int(pool_mode), int(score_mode), 0, _ptr(sl))
+    threads = _load().laq_oracle_evict_variant(
+        _ptr(q), _ptr(k), _ptr(v), NL, Bt, Hq, Hkv, D, L, W, R, kernel, B, scale, ctypes.byref(var),
+        _ptr(ul), 0 if ul is None else ul.shape[0], _ptr(scores), _ptr(colsum), _ptr(idx), _ptr(k_out),
         _ptr(v_out), 1 if fast_select else 0)
     out = {"scores": scores, "idx": idx, "k_out": k_out, "v_out": v_out, "threads": threads}
     if want_colsum:

@@ -391,3 +391,107 @@ def test_recall_hand_cases_and_numpy_intersection():
     small, big = orc.select(p, 500, 0, 50), orc.select(p, 500, 0, 200)
     assert orc.recall(big, small) == (1.0, 50)
     assert orc.recall(small, big)[1] == 50
+
+
+# ---------------------------------------------------------------- maximum pooling
+@pytest.mark.parametrize("kernel", [1, 3, 5, 7])
+def test_max_pool_matches_library_max_pool(kernel):
+    g = torch.Generator().manual_seed(43)
+    c = torch.rand(61, generator=g, dtype=torch.float64) - 0.3     # some negative values too
+    p = orc.pool(c.numpy(), 61, kernel, mode=1)
+    want = torch.nn.functional.max_pool1d(c[None, None], kernel, stride=1,
+                                          padding=kernel // 2)[0, 0].numpy()
+    assert (p == want).all()
+    if kernel == 1:
+        assert (p == c.numpy()).all()
+
+
+def test_max_pool_closed_forms_and_tail():
+    # a single spike becomes a plateau of width k; an increasing ramp is shifted by k/2
+    Ls, kernel = 30, 5
+    c = np.zeros(Ls)
+    c[11] = 2.5
+    p = orc.pool(c, Ls, kernel, mode=1)
+    assert p.tolist() == [2.5 if 9 <= j <= 13 else 0.0 for j in range(Ls)]
+    ramp = np.arange(Ls, dtype=np.float64)
+    p = orc.pool(ramp, Ls, kernel, mode=1)
+    assert p.tolist() == [float(min(j + 2, Ls - 1)) for j in range(Ls)]
+    # all values negative: padding must not contribute a zero
+    p = orc.pool(-1.0 - ramp, Ls, kernel, mode=1)
+    assert p.tolist() == [-1.0 - max(j - 2, 0) for j in range(Ls)]
+    # the retained tail is invisible to the pool
+    c2 = np.concatenate([ramp, np.full(6, 1e9)])
+    assert (orc.pool(c2, Ls, kernel, mode=1) == orc.pool(ramp, Ls, kernel, mode=1)).all()
+
+
+# ---------------------------------------------------------------- Eq. 4 read literally (raw logit sums)
+def test_rawsum_is_the_summed_query_times_keys():
+    G, W, D, L = 3, 5, 16, 37
+    q, k = rand_bf16((G, W, D), 51), rand_bf16((L, D), 52)
+    c = orc.unit_rawsum(q, k)
+    # another route: add the queries first, then one matrix-vector product
+    want = (k.double() @ q.double().reshape(-1, D).sum(0)).numpy() / math.sqrt(D)
+    np.testing.assert_allclose(c, want, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(orc.unit_rawsum(q, k, scale=0.5), want * 0.5 * math.sqrt(D),
+                               rtol=1e-12, atol=1e-13)
+    # odd in K, additive over query heads
+    np.testing.assert_allclose(orc.unit_rawsum(q, -k), -c, rtol=1e-15)
+    parts = sum(orc.unit_rawsum(q[g:g + 1], k) for g in range(G))
+    np.testing.assert_allclose(parts, c, rtol=1e-12, atol=1e-13)
+
+
+def test_rawsum_hand_example_small_integers():
+    # q rows (1,2) and (3,-1); keys (1,0), (0,1), (2,2): row sums of Q K^T = 4, 1, 10; scale 1/2
+    q = bf16(torch.tensor([[[1.0, 2.0], [3.0, -1.0]]]))
+    k = bf16(torch.tensor([[1.0, 0.0], [0.0, 1.0], [2.0, 2.0]]))
+    assert orc.unit_rawsum(q, k, scale=0.5).tolist() == [2.0, 0.5, 5.0]
+
+
+def test_evict_variants_raw_mode_and_max_pool():
+    NL, Bt, Hq, Hkv, D, L, W, kernel, B = 1, 2, 4, 2, 16, 80, 4, 3, 24
+    g = torch.Generator().manual_seed(14)
+    q = bf16(torch.randn((NL, Bt, Hq, W, D), generator=g))
+    k = bf16(torch.randn((NL, Bt, Hkv, L, D), generator=g))
+    v = bf16(torch.randn((NL, Bt, Hkv, L, D), generator=g))
+    R, G = W, Hq // Hkv
+    raw = orc.evict(q, k, v, R, 1, B, score_mode=1)
+    mx = orc.evict(q, k, v, R, kernel, B, pool_mode=1, want_colsum=True)
+    for b in range(Bt):
+        for h in range(Hkv):
+            s = (k[0, b, h].double() @ q[0, b, h * G:(h + 1) * G].double().reshape(-1, D).sum(0)) / math.sqrt(D)
+            np.testing.assert_allclose(raw["scores"][0, b, h], s[:L - R].numpy(), rtol=1e-12, atol=1e-13)
+            top = torch.topk(s[:L - R], B - R).indices.sort().values.tolist()
+            assert raw["idx"][0, b, h].tolist() == top + list(range(L - R, L))
+            want = torch.nn.functional.max_pool1d(torch.from_numpy(mx["colsum"][0, b, h][None, None, :L - R]),
+                                                  kernel, stride=1, padding=kernel // 2)[0, 0].numpy()
+            assert (mx["scores"][0, b, h] == want).all()
+            assert (mx["idx"][0, b, h] == orc.select(want, L, R, B)).all()
+
+
+# ---------------------------------------------------------------- prompts of different lengths
+def test_seq_lens_equal_separate_runs_on_truncated_prompts():
+    NL, Bt, Hq, Hkv, D, L, W, Wl, kernel, B = 2, 3, 4, 2, 16, 96, 6, 2, 5, 20
+    g = torch.Generator().manual_seed(15)
+    q = bf16(torch.randn((NL, Bt, Hq, W, D), generator=g))
+    k = bf16(torch.randn((NL, Bt, Hkv, L, D), generator=g))
+    v = bf16(torch.randn((NL, Bt, Hkv, L, D), generator=g))
+    lens = np.array([96, 41, 70], np.int32)
+    R = W
+    # rows beyond a prompt's length hold garbage that must never be read
+    k2, v2 = k.clone(), v.clone()
+    for b in range(Bt):
+        k2[:, b, :, lens[b]:] = float("nan")
+        v2[:, b, :, lens[b]:] = float("nan")
+    out = orc.evict(q, k2, v2, R, kernel, B, local_window=Wl, seq_lens=lens, want_colsum=True)
+    for b in range(Bt):
+        Lb = int(lens[b])
+        ref = orc.evict(q[:, b:b + 1], k[:, b:b + 1, :, :Lb], v[:, b:b + 1, :, :Lb], R, kernel, B,
+                        local_window=Wl, want_colsum=True)
+        assert (out["scores"][:, b, :, :Lb - R] == ref["scores"][:, 0]).all()
+        assert (out["scores"][:, b, :, Lb - R:] == 0).all()
+        assert (out["colsum"][:, b, :, :Lb] == ref["colsum"][:, 0]).all()
+        assert (out["colsum"][:, b, :, Lb:] == 0).all()
+        assert (out["idx"][:, b] == ref["idx"][:, 0]).all()
+        assert (out["idx"][:, b, :, B - R:] == np.arange(Lb - R, Lb)).all()
+        assert (out["k_out"][:, b] == ref["k_out"][:, 0]).all()
+        assert (out["v_out"][:, b] == ref["v_out"][:, 0]).all()
