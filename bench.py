@@ -50,6 +50,9 @@ def parse_args():
     ap.add_argument("--prompt-len", type=int, default=0, help="override the prompt length (profiling)")
     ap.add_argument("--local-window", type=int, default=0,
                     help="LAQ++ (Eq. 5): this many of the window's queries are causal local queries")
+    ap.add_argument("--score-mode", default="softmax", choices=["softmax", "raw"],
+                    help="raw = Eq. 4 read literally (sums of raw logits, one pass over K)")
+    ap.add_argument("--pool-mode", default="avg", choices=["avg", "max"])
     ap.add_argument("--tiles-per-task", type=int, default=0)
     ap.add_argument("--lag-units", type=int, default=0)
     return ap.parse_args()
@@ -271,6 +274,8 @@ def main():
     p = laq.params_for(q, k, cfg.keep_tail, cfg.pool_kernel, B, v=v, out=k_out)
     p.tiles_per_task, p.sched_lag_units = args.tiles_per_task, args.lag_units
     p.local_window = args.local_window
+    p.score_mode = laq.LAQ_SCORE_RAW if args.score_mode == "raw" else laq.LAQ_SCORE_SOFTMAX
+    p.pool_mode = laq.LAQ_POOL_MAX if args.pool_mode == "max" else laq.LAQ_POOL_AVG
     ws = laq.alloc_workspace(p, dev)
 
     def step():
@@ -317,8 +322,10 @@ def main():
     peak, peak_src = measured_peaks()
     score_bytes, gather_bytes = algorithmic_bytes(cfg, B)
     achieved = score_bytes / (score_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "score_tc_kernel", "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES,
+    raw = args.score_mode == "raw"
+    roofline = {"bound": "hbm", "kernel": "score_raw_d128_kernel" if raw else "score_tc_kernel",
+                "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "traffic": None if raw else NCU_TRAFFIC_BYTES,
                 "peak_source": peak_src, "algorithmic_bytes_per_launch": score_bytes,
                 "kernel_ms": score_ms, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
     # The scoring kernel's busiest unit is the MUFU: two base-2 exponentials per (row, key) pair
@@ -326,9 +333,10 @@ def main():
     n_exp = 2.0 * cfg.units * cfg.rows * cfg.prompt_len
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
     mufu_peak = 16.0 * sms * (clocks.get("sm_max_mhz") or 1965) * 1e6
-    roofline["mufu"] = {"bound": "alu", "achieved": n_exp / (score_ms * 1e-3), "peak": mufu_peak,
-                        "unit": "ex2/s", "frac": n_exp / (score_ms * 1e-3) / mufu_peak,
-                        "peak_source": "16 ex2 per clock and SM (measured) x SMs x max SM clock"}
+    if not raw:
+        roofline["mufu"] = {"bound": "alu", "achieved": n_exp / (score_ms * 1e-3), "peak": mufu_peak,
+                            "unit": "ex2/s", "frac": n_exp / (score_ms * 1e-3) / mufu_peak,
+                            "peak_source": "16 ex2 per clock and SM (measured) x SMs x max SM clock"}
     step_gbs = (score_bytes + gather_bytes) / (ms_per_step * 1e-3) / 1e9
     step_roofline = {"algorithmic_bytes_per_step": score_bytes + gather_bytes, "achieved": step_gbs,
                      "unit": "GB/s", "frac_of_measured": step_gbs / peak,
@@ -343,6 +351,8 @@ def main():
         torch.cuda.empty_cache()
         he = laq.HostEvictor(tuple(hq.shape), tuple(hk.shape), B, cfg.pool_kernel, cfg.keep_tail, dev)
         he.params.tiles_per_task, he.params.sched_lag_units = args.tiles_per_task, args.lag_units
+        he.params.local_window, he.params.score_mode, he.params.pool_mode = (
+            p.local_window, p.score_mode, p.pool_mode)
         he.run(hq, hk, hv)
         torch.cuda.synchronize()
         n_e2e = 3
@@ -371,7 +381,9 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-            "data": "synthetic", "config": config_dict(cfg, B),
+            "data": "synthetic",
+            "config": dict(config_dict(cfg, B), score_mode=args.score_mode, pool_mode=args.pool_mode,
+                           local_window=args.local_window),
             "kv_entries_per_s": cfg.units * cfg.prompt_len * world / (ms_per_step * 1e-3),
             "roofline": roofline, "step_roofline": step_roofline, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": launches_per_step * K, "clocks": clocks,

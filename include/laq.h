@@ -28,7 +28,8 @@
  *               column sums below run over the keys a row sees)
  *   2. softmax  P[r][j] = exp(s[r][j]-m_r) / l_r,  m_r = max_j s[r][j],  l_r = sum_j exp(s[r][j]-m_r)
  *   3. column sums  c[j] = sum_r P[r][j]
- *   4. pooling  p[j] = (1/k) * sum_{|t|<=k/2, 0<=j+t<Ls} c[j+t],  j in [0,Ls)   (zero padded)
+ *   4. pooling  p[j] = (1/k) * sum_{|t|<=k/2, 0<=j+t<Ls} c[j+t],  j in [0,Ls)   (zero padded;
+ *               or the maximum over the same window, see laq_pool_mode)
  *   5. top-k    the Kb positions of largest p (ties: lower position wins), written ascending,
  *               followed by the tail Ls..L-1
  *   6. gather   K_out[t] = K[idx[t]],  V_out[t] = V[idx[t]]
@@ -75,7 +76,16 @@ typedef enum {
   LAQ_ERR_INTERNAL = 6
 } laq_status;
 
-typedef enum { LAQ_POOL_AVG = 0 } laq_pool_mode;
+/* Step 4. LAQ_POOL_AVG: average over the k-wide window, zero padded, divisor always k (the pooling
+ * Section 5.1 names). LAQ_POOL_MAX: maximum over the window positions that exist (the other common
+ * choice of SnapKV-style eviction; not used by the paper's experiments). */
+typedef enum { LAQ_POOL_AVG = 0, LAQ_POOL_MAX = 1 } laq_pool_mode;
+
+/* Steps 2-3. LAQ_SCORE_SOFTMAX: column sums of the per-row softmax (attention weights), the
+ * reading used throughout. LAQ_SCORE_RAW: Eq. 4 taken literally, c[j] = sum_r s[r][j], the sum of
+ * the raw scaled logits over the window rows with no softmax (one pass over K; scores may be
+ * negative; local_window has no effect because it only masks positions inside the tail). */
+typedef enum { LAQ_SCORE_SOFTMAX = 0, LAQ_SCORE_RAW = 1 } laq_score_mode;
 
 /* Problem description. Plain data; copy freely. All strides are in bf16 ELEMENTS. */
 typedef struct {
@@ -100,7 +110,7 @@ typedef struct {
    * queries and see every prompt key. 0 = plain LAQ (Eq. 4). Needs local_window <= window_len and
    * local_window <= keep_tail, so that every scored position is visible to every query. */
   int32_t local_window;
-  int32_t reserved0;       /* must be 0 */
+  int32_t score_mode;      /* laq_score_mode */
   /* Q [NL][Bt][Hq][W][D] */
   int64_t q_stride_layer, q_stride_batch, q_stride_head, q_stride_pos;
   /* K [NL][Bt][Hkv][L][D] */
@@ -163,7 +173,7 @@ LAQ_API laq_status laq_score_static(const laq_params* p, const void* q, const vo
 /*
  * Step 5 (Eq. 4's ArgSort(...)[:B]): per unit, the B-R positions of largest score, ties to the
  * lower position, then the retained tail.
- *   scores  device, fp32, dense [NL][Bt][Hkv][L-R], every value >= 0 and not NaN
+ *   scores  device, fp32, dense [NL][Bt][Hkv][L-R], no NaN (negative values are allowed)
  *   idx     device, int32, dense [NL][Bt][Hkv][B]; first B-R entries strictly ascending in
  *           [0, L-R), last R entries are L-R .. L-1
  * Only n_layers, batch, n_kv_heads, prompt_len, keep_tail and budget of `p` are read.

@@ -22,6 +22,8 @@ LAQ_ERR_WORKSPACE = 3
 LAQ_ERR_CUDA = 4
 LAQ_ERR_TIMEOUT = 5
 LAQ_ERR_INTERNAL = 6
+LAQ_POOL_AVG, LAQ_POOL_MAX = 0, 1
+LAQ_SCORE_SOFTMAX, LAQ_SCORE_RAW = 0, 1
 
 EXPORTS = (
     "laq_params_dense_strides", "laq_workspace_bytes", "laq_score", "laq_select", "laq_compact",
@@ -38,7 +40,7 @@ class LaqParams(ctypes.Structure):
         "n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "prompt_len", "window_len",
         "keep_tail", "pool_kernel", "pool_mode", "budget")] + [("softmax_scale", ctypes.c_float),
         ("tiles_per_task", ctypes.c_int32), ("sched_lag_units", ctypes.c_int32),
-        ("local_window", ctypes.c_int32), ("reserved0", ctypes.c_int32)] + [
+        ("local_window", ctypes.c_int32), ("score_mode", ctypes.c_int32)] + [
         (f"{t}_stride_{d}", ctypes.c_int64) for t in ("q", "k", "v", "o")
         for d in ("layer", "batch", "head", "pos")]
 
@@ -235,7 +237,8 @@ def laq_version() -> int:
 
 def evict(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, budget: int, pool_kernel: int = 7,
           keep_tail: Optional[int] = None, want_scores: bool = False, ws=None, stream=None,
-          softmax_scale: float = 0.0, local_window: int = 0):
+          softmax_scale: float = 0.0, local_window: int = 0, pool_mode: int = 0,
+          score_mode: int = 0):
     """Convenience call: allocates the outputs with torch and runs ``laq_evict``.
 
     q [NL,Bt,Hq,W,D], k and v [NL,Bt,Hkv,L,D], bf16 CUDA tensors. Returns a dict with 'k_out',
@@ -253,6 +256,8 @@ def evict(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, budget: int, pool_k
     p = params_for(q, k, R, pool_kernel, budget, v=v, out=k_out)
     p.softmax_scale = softmax_scale  # 0 selects 1/sqrt(head_dim)
     p.local_window = local_window    # > 0: LAQ++ unified window (Eq. 5)
+    p.pool_mode = pool_mode          # LAQ_POOL_AVG / LAQ_POOL_MAX
+    p.score_mode = score_mode        # LAQ_SCORE_SOFTMAX / LAQ_SCORE_RAW (Eq. 4 read literally)
     if ws is None:
         ws = alloc_workspace(p, k.device)
     laq_evict(p, q, k, v, k_out, v_out, idx, scores, ws, stream)

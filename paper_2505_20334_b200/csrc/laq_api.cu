@@ -21,10 +21,11 @@ laq_status derive_dims(const laq_params* p, Dims* d) {
   if (p->pool_kernel < 1 || (p->pool_kernel % 2) == 0) return LAQ_ERR_INVALID_ARG;
   if (!(p->softmax_scale >= 0.0f) || isinf(p->softmax_scale)) return LAQ_ERR_INVALID_ARG;
   if (p->tiles_per_task < 0 || p->sched_lag_units < 0) return LAQ_ERR_INVALID_ARG;
-  if (p->local_window < 0 || p->local_window > p->window_len || p->local_window > p->keep_tail ||
-      p->reserved0 != 0)
+  if (p->local_window < 0 || p->local_window > p->window_len || p->local_window > p->keep_tail)
     return LAQ_ERR_INVALID_ARG;
-  if (p->pool_mode != LAQ_POOL_AVG) return LAQ_ERR_UNSUPPORTED;
+  if ((p->pool_mode != LAQ_POOL_AVG && p->pool_mode != LAQ_POOL_MAX) ||
+      (p->score_mode != LAQ_SCORE_SOFTMAX && p->score_mode != LAQ_SCORE_RAW))
+    return LAQ_ERR_INVALID_ARG;
   if ((p->head_dim % 8) != 0 || p->head_dim > 256) return LAQ_ERR_UNSUPPORTED;
   const int64_t M = (int64_t)(p->n_q_heads / p->n_kv_heads) * p->window_len;
   if (M > 256) return LAQ_ERR_UNSUPPORTED;
@@ -37,6 +38,8 @@ laq_status derive_dims(const laq_params* p, Dims* d) {
   d->L = p->prompt_len;
   d->W = p->window_len;
   d->W_local = p->local_window;
+  d->pool_max = p->pool_mode == LAQ_POOL_MAX;
+  d->score_raw = p->score_mode == LAQ_SCORE_RAW;
   d->R = p->keep_tail;
   d->kpool = p->pool_kernel;
   d->B = p->budget;
@@ -97,6 +100,8 @@ void plan_workspace(const Dims& d, int tiles_per_task, Workspace* w) {
   off = align_up(off + (size_t)d.U * w->n_part * w->M_pad * sizeof(float2), 256);
   w->off_rowoff = off;
   off = align_up(off + (size_t)d.U * w->M_pad * sizeof(float), 256);
+  w->off_qsum = off;
+  if (d.score_raw) off = align_up(off + (size_t)d.U * d.D * sizeof(float), 256);
   w->off_colsum = off;
   off = align_up(off + (size_t)d.U * w->L_pad * sizeof(float), 256);
   w->off_pooled = off;
@@ -119,7 +124,8 @@ static laq_status run_scoring(const laq_params* p, const Dims& d, const Workspac
   if (cudaMemsetAsync(ws + w.off_hdr, 0, w.off_part - w.off_hdr, stream) != cudaSuccess)
     return LAQ_ERR_CUDA;
   if (g_ev_begin && cudaEventRecord(g_ev_begin, stream) != cudaSuccess) return LAQ_ERR_CUDA;
-  const laq_status st = use_tensor_core_path(d)
+  const laq_status st = d.score_raw ? score_raw_launch(*p, d, w, q, k, ws, stream, launches)
+                        : use_tensor_core_path(d)
                             ? score_tc_launch(*p, d, w, q, k, ws, stream, launches)
                             : score_simt_launch(*p, d, w, q, k, ws, stream, launches);
   if (g_ev_end && cudaEventRecord(g_ev_end, stream) != cudaSuccess) return LAQ_ERR_CUDA;

@@ -12,6 +12,8 @@ namespace laq {
 struct Dims {
   int NL, Bt, Hq, Hkv, G, D, L, W, R, kpool, B;
   int W_local;  // leading causal queries of each head's window (LAQ++), 0 for plain LAQ
+  int pool_max;   // 1: maximum pooling, 0: average pooling
+  int score_raw;  // 1: raw logit sums (Eq. 4 read literally), 0: softmax column sums
   int M;        // G*W softmax rows per unit
   int Ls, Kb;   // scored positions, selected slots
   int64_t U;    // units
@@ -24,11 +26,12 @@ struct Dims {
 //   unit_cnt : int32 [U]   partial row statistics delivered so far, zeroed per call
 //   part     : float2 [U][n_part][M_pad]  partial (max, sum) in the log2 domain, one per task
 //   row_off  : float [U][M_pad]  b_r = log2e*scale*m_r + log2(l_r) (CUDA-core path only)
+//   qsum     : float [U][D]  sum of the unit's query rows (raw-logit mode only)
 //   colsum   : float [U][L_pad]  c_j (step 3)
 //   pooled   : float [U][Ls]     p_j (step 4) when the caller gave no scores buffer
 //   idx      : int32 [U][B]      kept positions when the caller gave no idx buffer
 struct Workspace {
-  size_t off_hdr, off_cnt, off_part, off_rowoff, off_colsum, off_pooled, off_idx, total;
+  size_t off_hdr, off_cnt, off_part, off_rowoff, off_qsum, off_colsum, off_pooled, off_idx, total;
   int n_part;  // partial-statistics slots per unit = scoring tasks per unit and sweep
   int M_pad;   // rows padded to a multiple of 32
   int L_pad;   // L padded to a multiple of 128
@@ -47,6 +50,9 @@ int choose_tiles_per_task(const Dims& d);
 // Tensor-core path (tcgen05 + TMA), head_dim 128, M <= 256.
 laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& w, const void* q,
                            const void* k, char* ws, cudaStream_t stream, int* launches);
+// Raw-logit mode (Eq. 4 read literally): one streaming pass over K on CUDA cores.
+laq_status score_raw_launch(const laq_params& p, const Dims& d, const Workspace& w, const void* q,
+                            const void* k, char* ws, cudaStream_t stream, int* launches);
 // CUDA-core path for every other shape.
 laq_status score_simt_launch(const laq_params& p, const Dims& d, const Workspace& w,
                              const void* q, const void* k, char* ws, cudaStream_t stream,

@@ -70,8 +70,9 @@ extern "C" laq_status laq_score_static(const laq_params* p, const void* q, const
   if (cudaMemsetAsync(ws + w.off_hdr, 0, w.off_part - w.off_hdr, stream) != cudaSuccess)
     return LAQ_ERR_CUDA;
   int launches = 0;
-  st = (d.D == 128 && d.M <= 256) ? score_tc_launch(*p, d, w, q, k, ws, stream, &launches)
-                                  : score_simt_launch(*p, d, w, q, k, ws, stream, &launches);
+  st = d.score_raw                  ? score_raw_launch(*p, d, w, q, k, ws, stream, &launches)
+       : (d.D == 128 && d.M <= 256) ? score_tc_launch(*p, d, w, q, k, ws, stream, &launches)
+                                    : score_simt_launch(*p, d, w, q, k, ws, stream, &launches);
   if (st != LAQ_OK) return st;
   return pool_launch(d, (const float*)(ws + w.off_colsum), w.L_pad, scores, stream, &launches);
 }

@@ -1,4 +1,4 @@
-// Step 4 (average pooling of the column sums) and step 5 (Eq. 4's ArgSort(...)[:B]: per-unit
+// Step 4 (average or maximum pooling of the column sums) and step 5 (Eq. 4's ArgSort(...)[:B]: per-unit
 // top-k by radix select on the fp32 bit patterns, ties to the lower position, ascending output
 // followed by the retained tail).
 #include "laq_internal.cuh"
@@ -9,20 +9,33 @@ namespace {
 constexpr int kSelThreads = 1024;
 constexpr int kSelWarps = kSelThreads / 32;
 
-// p_j = (1/k) * sum_{|t| <= k/2, 0 <= j+t < Ls} c_{j+t}: zero padding, divisor always k.
-__global__ void pool_kernel(const float* __restrict__ colsum, int L_pad, float* __restrict__ pooled,
-                            int Ls, int kpool, float inv_k) {
-  const int64_t u = blockIdx.y;
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= Ls) return;
-  const float* c = colsum + u * L_pad;
-  const int h = kpool / 2;
+// Average pooling: p_j = (1/k) * sum_{|t| <= k/2, 0 <= j+t < Ls} c_{j+t} (zero padding, divisor
+// always k). Maximum pooling: the largest c_{j+t} over the same window positions that exist.
+// One position near an edge of [0, Ls), or any position when the window is not unrolled.
+__device__ __forceinline__ float pool_at(const float* c, int j, int h, int Ls, float inv_k,
+                                         int pool_max) {
+  if (pool_max) {
+    float best = c[j];
+    for (int t = -h; t <= h; ++t) {
+      const int jj = j + t;
+      if (jj >= 0 && jj < Ls) best = fmaxf(best, c[jj]);
+    }
+    return best;
+  }
   float acc = 0.f;
   for (int t = -h; t <= h; ++t) {
     const int jj = j + t;
     if (jj >= 0 && jj < Ls) acc += c[jj];
   }
-  pooled[u * Ls + j] = acc * inv_k;
+  return acc * inv_k;
+}
+
+__global__ void pool_kernel(const float* __restrict__ colsum, int L_pad, float* __restrict__ pooled,
+                            int Ls, int kpool, float inv_k, int pool_max) {
+  const int64_t u = blockIdx.y;
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= Ls) return;
+  pooled[u * Ls + j] = pool_at(colsum + u * L_pad, j, kpool / 2, Ls, inv_k, pool_max);
 }
 
 // Order-preserving map from fp32 bits to uint32 (larger float <=> larger key).
@@ -146,18 +159,13 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const float* _
                                                                   int L_pad, float* pooled_out,
                                                                   int32_t* __restrict__ idx, int Ls,
                                                                   int Kb, int R, int B, int kpool,
-                                                                  float inv_k) {
+                                                                  float inv_k, int pool_max) {
   extern __shared__ float s_pooled[];
   const int64_t u = blockIdx.x;
   const float* c = colsum + u * (int64_t)L_pad;
   const int h = kpool / 2;
   for (int j = threadIdx.x; j < Ls; j += kSelThreads) {
-    float acc = 0.f;
-    for (int t = -h; t <= h; ++t) {
-      const int jj = j + t;
-      if (jj >= 0 && jj < Ls) acc += c[jj];
-    }
-    const float pj = acc * inv_k;
+    const float pj = pool_at(c, j, h, Ls, inv_k, pool_max);
     s_pooled[j] = pj;
     if (pooled_out) pooled_out[u * (int64_t)Ls + j] = pj;
   }
@@ -199,7 +207,7 @@ __device__ __forceinline__ void transpose32(uint32_t (&a)[32]) {
 template <int kPoolStatic>
 __global__ void __launch_bounds__(kSelThreads) pool_select_reg_kernel(
     const float* __restrict__ colsum, int L_pad, float* pooled_out, int32_t* __restrict__ idx, int Ls,
-    int Kb, int R, int B, int kpool, float inv_k) {
+    int Kb, int R, int B, int kpool, float inv_k, int pool_max) {
   __shared__ uint32_t s_cnt[2][kSelWarps];
   __shared__ uint32_t s_gt[kSelWarps], s_eq[kSelWarps];
   const int64_t u = blockIdx.x;
@@ -216,21 +224,22 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_reg_kernel(
     const int j = base + it * 32;
     uint32_t key = 0u;
     if (j < Ls) {
-      float acc = 0.f;
-      if (j >= h && j + h < Ls) {
-        if (kPoolStatic > 0) {
+      float pj;
+      if (kPoolStatic > 0 && j >= h && j + h < Ls) {
+        // interior position, window unrolled
+        if (pool_max) {
+          pj = c[j];
+#pragma unroll
+          for (int t = -(kPoolStatic / 2); t <= kPoolStatic / 2; ++t) pj = fmaxf(pj, c[j + t]);
+        } else {
+          float acc = 0.f;
 #pragma unroll
           for (int t = -(kPoolStatic / 2); t <= kPoolStatic / 2; ++t) acc += c[j + t];
-        } else {
-          for (int t = -h; t <= h; ++t) acc += c[j + t];
+          pj = acc * inv_k;
         }
       } else {
-        for (int t = -h; t <= h; ++t) {
-          const int jj = j + t;
-          if (jj >= 0 && jj < Ls) acc += c[jj];
-        }
+        pj = pool_at(c, j, h, Ls, inv_k, pool_max);
       }
-      const float pj = acc * inv_k;
       if (pooled_out) pooled_out[u * (int64_t)Ls + j] = pj;
       key = order_key(pj);
       alive |= 1u << it;
@@ -301,12 +310,13 @@ laq_status pool_launch(const Dims& d, const float* colsum, int L_pad, float* poo
     for (int64_t u0 = 0; u0 < d.U; u0 += 65535) {
       const unsigned nu = (unsigned)((d.U - u0 < 65535) ? d.U - u0 : 65535);
       pool_kernel<<<dim3((d.Ls + 255) / 256, nu), 256, 0, stream>>>(
-          colsum + u0 * L_pad, L_pad, pooled + u0 * d.Ls, d.Ls, d.kpool, 1.0f / (float)d.kpool);
+          colsum + u0 * L_pad, L_pad, pooled + u0 * d.Ls, d.Ls, d.kpool, 1.0f / (float)d.kpool,
+          d.pool_max);
       *launches += 1;
     }
   } else {
     pool_kernel<<<dim3((d.Ls + 255) / 256, (unsigned)d.U), 256, 0, stream>>>(
-        colsum, L_pad, pooled, d.Ls, d.kpool, 1.0f / (float)d.kpool);
+        colsum, L_pad, pooled, d.Ls, d.kpool, 1.0f / (float)d.kpool, d.pool_max);
     *launches += 1;
   }
   return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;
@@ -329,7 +339,8 @@ laq_status pool_select_launch(const Dims& d, const float* colsum, int L_pad, flo
     const unsigned grid = (unsigned)d.U;
 #define LAQ_LAUNCH_POOL_SELECT(KP)                                                         \
   pool_select_reg_kernel<KP><<<grid, kSelThreads, 0, stream>>>(colsum, L_pad, pooled_out, idx, \
-                                                               d.Ls, d.Kb, d.R, d.B, d.kpool, inv_k)
+                                                               d.Ls, d.Kb, d.R, d.B, d.kpool, inv_k, \
+                                                               d.pool_max)
     switch (d.kpool) {
       case 1: LAQ_LAUNCH_POOL_SELECT(1); break;
       case 3: LAQ_LAUNCH_POOL_SELECT(3); break;
@@ -348,7 +359,8 @@ laq_status pool_select_launch(const Dims& d, const float* colsum, int L_pad, flo
                            (int)smem) != cudaSuccess)
     return LAQ_ERR_CUDA;
   pool_select_kernel<<<(unsigned)d.U, kSelThreads, smem, stream>>>(
-      colsum, L_pad, pooled_out, idx, d.Ls, d.Kb, d.R, d.B, d.kpool, 1.0f / (float)d.kpool);
+      colsum, L_pad, pooled_out, idx, d.Ls, d.Kb, d.R, d.B, d.kpool, 1.0f / (float)d.kpool,
+      d.pool_max);
   *launches += 1;
   *done = true;
   return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;

@@ -28,17 +28,18 @@ def rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed, kscale=1.0):
     return q, k, v
 
 
-def run_evict(laq, q, k, v, R, kernel, B, local_window=0):
+def run_evict(laq, q, k, v, R, kernel, B, local_window=0, pool_mode=0, score_mode=0):
     out = laq.evict(q.cuda(), k.cuda(), v.cuda(), B, pool_kernel=kernel, keep_tail=R,
-                    want_scores=True, local_window=local_window)
+                    want_scores=True, local_window=local_window, pool_mode=pool_mode,
+                    score_mode=score_mode)
     assert laq.laq_last_device_status(out["params"], out["ws"]) == laq.LAQ_OK
     return out
 
 
-def compare_all_units(laq, q, k, v, R, kernel, B, out=None, local_window=0):
+def compare_all_units(laq, q, k, v, R, kernel, B, out=None, local_window=0, pool_mode=0):
     """Full comparison of every unit of a (small) problem against the oracle."""
-    out = out or run_evict(laq, q, k, v, R, kernel, B, local_window)
-    ref = orc.evict(q, k, v, R, kernel, B, local_window=local_window)
+    out = out or run_evict(laq, q, k, v, R, kernel, B, local_window, pool_mode)
+    ref = orc.evict(q, k, v, R, kernel, B, local_window=local_window, pool_mode=pool_mode)
     NL, Bt, Hkv, L = k.shape[0], k.shape[1], k.shape[2], k.shape[3]
     got_scores = out["scores"].cpu().numpy()
     err = score_rel_err(got_scores, ref["scores"])
@@ -217,6 +218,65 @@ def test_unified_window_matches_oracle(laq, shape):
     plain = run_evict(laq, q, k, v, W, kernel, B)
     masked = run_evict(laq, q, k, v, W, kernel, B, local_window=Wl)
     assert not torch.allclose(plain["scores"], masked["scores"], rtol=1e-3, atol=0)
+
+
+VARIANT_SHAPES = [
+    # NL Bt Hq Hkv D    L     W  k  B
+    (1, 2, 8, 2, 128, 1300, 16, 7, 150),   # M = 64, ragged last tile
+    (1, 1, 4, 1, 128, 4500, 32, 5, 300),   # M = 128, several key chunks of the raw pass
+    (1, 1, 8, 2, 64, 500, 8, 3, 90),       # head_dim 64
+]
+
+
+@pytest.mark.parametrize("shape", VARIANT_SHAPES, ids=[f"L{s[5]}-D{s[4]}-k{s[7]}" for s in VARIANT_SHAPES])
+def test_max_pooling_matches_oracle(laq, shape):
+    NL, Bt, Hq, Hkv, D, L, W, kernel, B = shape
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=L + kernel, kscale=1.5)
+    err, _ = compare_all_units(laq, q, k, v, W, kernel, B, pool_mode=1)
+    assert err < SCORE_RTOL
+    avg = run_evict(laq, q, k, v, W, kernel, B)
+    mx = run_evict(laq, q, k, v, W, kernel, B, pool_mode=1)
+    assert (mx["scores"] >= avg["scores"]).all() and not torch.equal(mx["scores"], avg["scores"])
+
+
+@pytest.mark.parametrize("shape", VARIANT_SHAPES, ids=[f"L{s[5]}-D{s[4]}-k{s[7]}" for s in VARIANT_SHAPES])
+def test_raw_logit_mode_matches_oracle(laq, shape):
+    # Eq. 4 read literally: sums of raw logits. The sums cancel, so the error is measured against
+    # the sum of the absolute terms: fp32 accumulation of D products and of M query rows stays
+    # below 2e-5 of it (D * 2^-24 = 7.6e-6 for the dot product, plus the query sum).
+    NL, Bt, Hq, Hkv, D, L, W, kernel, B = shape
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=3 * L + 1)
+    R, G = W, Hq // Hkv
+    out = run_evict(laq, q, k, v, R, kernel, B, score_mode=1)
+    ref = orc.evict(q, k, v, R, kernel, B, score_mode=1)
+    got_scores, got_idx = out["scores"].cpu().numpy(), out["idx"].cpu().numpy()
+    kb, vb, ko, vo = bits(k), bits(v), bits(out["k_out"]), bits(out["v_out"])
+    for n in range(NL):
+        for b in range(Bt):
+            for h in range(Hkv):
+                qs = q[n, b, h * G:(h + 1) * G].double().reshape(-1, D).sum(0)
+                mag = ((k[n, b, h].double().abs() @ qs.abs()) / np.sqrt(D)).numpy()
+                tol = 2e-5 * orc.pool(mag, L - R, kernel)      # the pool averages the bounds too
+                ref_p = ref["scores"][n, b, h]
+                assert (np.abs(got_scores[n, b, h] - ref_p) <= tol).all()
+                # kept set: equal to the oracle's except where the score is within the error of
+                # the oracle's Kb-th largest
+                theta = np.sort(ref_p)[::-1][B - R - 1]
+                diff = sorted(set(got_idx[n, b, h, :B - R].tolist()) ^ set(ref["idx"][n, b, h, :B - R].tolist()))
+                assert all(abs(ref_p[j] - theta) <= 2 * tol.max() for j in diff)
+                assert got_idx[n, b, h, B - R:].tolist() == list(range(L - R, L))
+                want = orc.select(got_scores[n, b, h], L, R, B, sorted_variant=True)
+                assert (got_idx[n, b, h] == want).all()            # negative scores order correctly
+                assert (ko[n, b, h] == kb[n, b, h][got_idx[n, b, h]]).all()
+                assert (vo[n, b, h] == vb[n, b, h][got_idx[n, b, h]]).all()
+    assert (got_scores < 0).any() and (got_scores > 0).any()
+
+
+def test_variant_argument_checks(laq):
+    q, k, v = rand_inputs(1, 1, 4, 2, 128, 300, 8, seed=4)
+    for kw in ({"pool_mode": 2}, {"pool_mode": -1}, {"score_mode": 2}):
+        with pytest.raises(laq.LaqError):
+            laq.evict(q.cuda(), k.cuda(), v.cuda(), 40, **kw)
 
 
 def test_local_window_argument_checks(laq):
