@@ -53,8 +53,11 @@ def parse_args():
     ap.add_argument("--score-mode", default="softmax", choices=["softmax", "raw"],
                     help="raw = Eq. 4 read literally (sums of raw logits, one pass over K)")
     ap.add_argument("--pool-mode", default="avg", choices=["avg", "max"])
+    ap.add_argument("--ragged", action="store_true",
+                    help="prompt b of the batch holds only L*(b+1)/batch positions (per-prompt lengths)")
+    ap.add_argument("--seq-lens", default="", help="explicit per-prompt lengths, comma separated")
     ap.add_argument("--tiles-per-task", type=int, default=0)
-    ap.add_argument("--lag-units", type=int, default=0)
+    ap.add_argument("--lag-tasks", type=int, default=0)
     return ap.parse_args()
 
 
@@ -148,11 +151,11 @@ def workload(args):
     return cfg
 
 
-def algorithmic_bytes(cfg, B):
+def algorithmic_bytes(cfg, B, mean_len=None):
     """Bytes the method must move per step: K once + Q for scoring; kept K/V rows read and written,
     the kept positions written (fp32 column sums and a second K sweep are overhead, not counted)."""
     D2 = 2 * cfg.head_dim
-    score = cfg.units * (D2 * cfg.prompt_len + D2 * cfg.rows)
+    score = cfg.units * (D2 * (cfg.prompt_len if mean_len is None else mean_len) + D2 * cfg.rows)
     gather = cfg.units * (2 * D2 * B + 2 * D2 * B + 4 * B)
     return score, gather
 
@@ -272,10 +275,15 @@ def main():
     v_out = torch.empty_like(k_out)
     idx = torch.empty((NL, Bt, Hkv, B), dtype=torch.int32, device=dev)
     p = laq.params_for(q, k, cfg.keep_tail, cfg.pool_kernel, B, v=v, out=k_out)
-    p.tiles_per_task, p.sched_lag_units = args.tiles_per_task, args.lag_units
+    p.tiles_per_task, p.sched_lag_tasks = args.tiles_per_task, args.lag_tasks
     p.local_window = args.local_window
     p.score_mode = laq.LAQ_SCORE_RAW if args.score_mode == "raw" else laq.LAQ_SCORE_SOFTMAX
     p.pool_mode = laq.LAQ_POOL_MAX if args.pool_mode == "max" else laq.LAQ_POOL_AVG
+    lens = [max(B + 1, L * (b + 1) // Bt) for b in range(Bt)] if args.ragged else None
+    if args.seq_lens:
+        lens = [int(x) for x in args.seq_lens.split(",")]
+    p.set_seq_lens(lens)
+    tokens_per_step = sum(lens) if lens else Bt * L
     ws = laq.alloc_workspace(p, dev)
 
     def step():
@@ -317,10 +325,10 @@ def main():
 
     total_ms = multi.max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / K
-    value = multi.whole_job_tokens_per_s(cfg.batch * cfg.prompt_len, world, ms_per_step)
+    value = multi.whole_job_tokens_per_s(tokens_per_step, world, ms_per_step)
 
     peak, peak_src = measured_peaks()
-    score_bytes, gather_bytes = algorithmic_bytes(cfg, B)
+    score_bytes, gather_bytes = algorithmic_bytes(cfg, B, tokens_per_step / Bt)
     achieved = score_bytes / (score_ms * 1e-3) / 1e9
     raw = args.score_mode == "raw"
     roofline = {"bound": "hbm", "kernel": "score_raw_d128_kernel" if raw else "score_tc_kernel",
@@ -330,7 +338,7 @@ def main():
                 "kernel_ms": score_ms, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
     # The scoring kernel's busiest unit is the MUFU: two base-2 exponentials per (row, key) pair
     # (one per sweep) at 16 per clock and SM.
-    n_exp = 2.0 * cfg.units * cfg.rows * cfg.prompt_len
+    n_exp = 2.0 * NL * Hkv * cfg.rows * tokens_per_step
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
     mufu_peak = 16.0 * sms * (clocks.get("sm_max_mhz") or 1965) * 1e6
     if not raw:
@@ -350,9 +358,10 @@ def main():
         del inputs, q, k, v, k_out, v_out
         torch.cuda.empty_cache()
         he = laq.HostEvictor(tuple(hq.shape), tuple(hk.shape), B, cfg.pool_kernel, cfg.keep_tail, dev)
-        he.params.tiles_per_task, he.params.sched_lag_units = args.tiles_per_task, args.lag_units
+        he.params.tiles_per_task, he.params.sched_lag_tasks = args.tiles_per_task, args.lag_tasks
         he.params.local_window, he.params.score_mode, he.params.pool_mode = (
             p.local_window, p.score_mode, p.pool_mode)
+        he.params.set_seq_lens(lens)
         he.run(hq, hk, hv)
         torch.cuda.synchronize()
         n_e2e = 3
@@ -364,7 +373,7 @@ def main():
         torch.cuda.synchronize()
         e2e_ms = s2.elapsed_time(e2) / n_e2e
         same = bool((he.h_idx.to(dev) == idx).all().item())
-        e2e = {"value": cfg.batch * cfg.prompt_len / (e2e_ms * 1e-3), "unit": UNIT,
+        e2e = {"value": tokens_per_step / (e2e_ms * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": he.h2d_bytes, "d2h_bytes_per_step": he.d2h_bytes,
                "ms_per_step": e2e_ms, "steps": n_e2e, "api": "laq_evict_host",
                "matches_device_run": same}
@@ -383,8 +392,8 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
             "config": dict(config_dict(cfg, B), score_mode=args.score_mode, pool_mode=args.pool_mode,
-                           local_window=args.local_window),
-            "kv_entries_per_s": cfg.units * cfg.prompt_len * world / (ms_per_step * 1e-3),
+                           local_window=args.local_window, seq_lens=lens),
+            "kv_entries_per_s": NL * Hkv * tokens_per_step * world / (ms_per_step * 1e-3),
             "roofline": roofline, "step_roofline": step_roofline, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": launches_per_step * K, "clocks": clocks,
         }))

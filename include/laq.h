@@ -103,7 +103,7 @@ typedef struct {
   float softmax_scale; /* 0 selects 1/sqrt(head_dim) */
   /* Scheduling knobs of the scoring kernel; 0 lets the library choose. */
   int32_t tiles_per_task;  /* 128-key tiles per scoring task (a task = one sweep over a key chunk) */
-  int32_t sched_lag_units; /* how many units the column-sum sweep trails the statistics sweep */
+  int32_t sched_lag_tasks; /* how many tasks the column-sum sweep trails the statistics sweep */
   /* LAQ++ (Eq. 5, unified window W u Q): the first local_window of each head's window_len queries
    * are the queries of the last local_window prompt positions (query i at position
    * L - local_window + i) and attend causally, to positions <= their own; the rest are lookahead
@@ -119,7 +119,18 @@ typedef struct {
   int64_t v_stride_layer, v_stride_batch, v_stride_head, v_stride_pos;
   /* K_out and V_out [NL][Bt][Hkv][B][D] (the same strides serve both) */
   int64_t o_stride_layer, o_stride_batch, o_stride_head, o_stride_pos;
+  /* Prompts of different lengths in one batch (the paper evaluates one prompt at a time; a
+   * serving batch is ragged). NULL: every prompt holds prompt_len positions. Otherwise a HOST
+   * array of `batch` int32, read during the call only: prompt b holds its first seq_lens[b]
+   * positions of the L allocated ones, budget < seq_lens[b] <= prompt_len, and batch <=
+   * LAQ_MAX_RAGGED_BATCH. Everything is then relative to that length Lb: keys [0, Lb), local
+   * queries at the last local_window of them, scored positions [0, Lb-R), tail [Lb-R, Lb). Rows of
+   * K and V beyond Lb are never used (they may hold anything); scores beyond Lb-R are written
+   * as 0. The tensors keep their [.. L ..] shapes and strides. */
+  const int32_t* seq_lens;
 } laq_params;
+
+#define LAQ_MAX_RAGGED_BATCH 512
 
 /* Fills the stride fields of `p` for densely packed tensors in the index order shown above. */
 LAQ_API void laq_params_dense_strides(laq_params* p);
@@ -175,8 +186,8 @@ LAQ_API laq_status laq_score_static(const laq_params* p, const void* q, const vo
  * lower position, then the retained tail.
  *   scores  device, fp32, dense [NL][Bt][Hkv][L-R], no NaN (negative values are allowed)
  *   idx     device, int32, dense [NL][Bt][Hkv][B]; first B-R entries strictly ascending in
- *           [0, L-R), last R entries are L-R .. L-1
- * Only n_layers, batch, n_kv_heads, prompt_len, keep_tail and budget of `p` are read.
+ *           [0, L-R), last R entries are L-R .. L-1 (with seq_lens: Lb in place of L)
+ * Only n_layers, batch, n_kv_heads, prompt_len, keep_tail, budget and seq_lens of `p` are read.
  */
 LAQ_API laq_status laq_select(const laq_params* p, const float* scores, int32_t* idx, void* cuda_stream);
 

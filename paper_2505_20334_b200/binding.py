@@ -39,10 +39,23 @@ class LaqParams(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "prompt_len", "window_len",
         "keep_tail", "pool_kernel", "pool_mode", "budget")] + [("softmax_scale", ctypes.c_float),
-        ("tiles_per_task", ctypes.c_int32), ("sched_lag_units", ctypes.c_int32),
+        ("tiles_per_task", ctypes.c_int32), ("sched_lag_tasks", ctypes.c_int32),
         ("local_window", ctypes.c_int32), ("score_mode", ctypes.c_int32)] + [
         (f"{t}_stride_{d}", ctypes.c_int64) for t in ("q", "k", "v", "o")
-        for d in ("layer", "batch", "head", "pos")]
+        for d in ("layer", "batch", "head", "pos")] + [("seq_lens", ctypes.POINTER(ctypes.c_int32))]
+
+    def set_seq_lens(self, lens) -> None:
+        """Per-prompt lengths (a sequence of `batch` ints, or None). The host array the C struct
+        points to is kept alive by this object."""
+        if lens is None:
+            self._seq_lens_buf = None
+            self.seq_lens = ctypes.POINTER(ctypes.c_int32)()
+            return
+        lens = [int(x) for x in lens]
+        if len(lens) != self.batch:
+            raise ValueError("seq_lens: one length per batch item is required")
+        self._seq_lens_buf = (ctypes.c_int32 * len(lens))(*lens)
+        self.seq_lens = ctypes.cast(self._seq_lens_buf, ctypes.POINTER(ctypes.c_int32))
 
 
 class LaqError(RuntimeError):
@@ -238,7 +251,7 @@ def laq_version() -> int:
 def evict(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, budget: int, pool_kernel: int = 7,
           keep_tail: Optional[int] = None, want_scores: bool = False, ws=None, stream=None,
           softmax_scale: float = 0.0, local_window: int = 0, pool_mode: int = 0,
-          score_mode: int = 0):
+          score_mode: int = 0, seq_lens=None):
     """Convenience call: allocates the outputs with torch and runs ``laq_evict``.
 
     q [NL,Bt,Hq,W,D], k and v [NL,Bt,Hkv,L,D], bf16 CUDA tensors. Returns a dict with 'k_out',
@@ -258,6 +271,7 @@ def evict(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, budget: int, pool_k
     p.local_window = local_window    # > 0: LAQ++ unified window (Eq. 5)
     p.pool_mode = pool_mode          # LAQ_POOL_AVG / LAQ_POOL_MAX
     p.score_mode = score_mode        # LAQ_SCORE_SOFTMAX / LAQ_SCORE_RAW (Eq. 4 read literally)
+    p.set_seq_lens(seq_lens)         # prompts of different lengths in one batch
     if ws is None:
         ws = alloc_workspace(p, k.device)
     laq_evict(p, q, k, v, k_out, v_out, idx, scores, ws, stream)

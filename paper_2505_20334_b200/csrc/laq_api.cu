@@ -10,6 +10,20 @@ namespace laq {
 static bool mult8(int64_t x) { return x > 0 && (x % 8) == 0; }
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Validates and copies the per-prompt lengths (budget < Lb <= L for every prompt).
+static laq_status derive_seq_lens(const laq_params* p, SeqLens* sl) {
+  sl->n = 0;
+  if (!p->seq_lens) return LAQ_OK;
+  if (p->batch > LAQ_MAX_RAGGED_BATCH) return LAQ_ERR_UNSUPPORTED;
+  for (int b = 0; b < p->batch; ++b) {
+    const int32_t len = p->seq_lens[b];
+    if (len <= p->budget || len > p->prompt_len) return LAQ_ERR_INVALID_ARG;
+    sl->len[b] = len;
+  }
+  sl->n = p->batch;
+  return LAQ_OK;
+}
+
 laq_status derive_dims(const laq_params* p, Dims* d) {
   if (!p) return LAQ_ERR_INVALID_ARG;
   if (p->n_layers < 1 || p->batch < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1 ||
@@ -20,7 +34,7 @@ laq_status derive_dims(const laq_params* p, Dims* d) {
     return LAQ_ERR_INVALID_ARG;
   if (p->pool_kernel < 1 || (p->pool_kernel % 2) == 0) return LAQ_ERR_INVALID_ARG;
   if (!(p->softmax_scale >= 0.0f) || isinf(p->softmax_scale)) return LAQ_ERR_INVALID_ARG;
-  if (p->tiles_per_task < 0 || p->sched_lag_units < 0) return LAQ_ERR_INVALID_ARG;
+  if (p->tiles_per_task < 0 || p->sched_lag_tasks < 0) return LAQ_ERR_INVALID_ARG;
   if (p->local_window < 0 || p->local_window > p->window_len || p->local_window > p->keep_tail)
     return LAQ_ERR_INVALID_ARG;
   if ((p->pool_mode != LAQ_POOL_AVG && p->pool_mode != LAQ_POOL_MAX) ||
@@ -48,9 +62,9 @@ laq_status derive_dims(const laq_params* p, Dims* d) {
   d->Kb = d->B - d->R;
   d->U = (int64_t)d->NL * d->Bt * d->Hkv;
   d->tiles_per_task = p->tiles_per_task;
-  d->sched_lag_units = p->sched_lag_units;
+  d->sched_lag_tasks = p->sched_lag_tasks;
   d->scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / sqrtf((float)d->D);
-  return LAQ_OK;
+  return derive_seq_lens(p, &d->sl);
 }
 
 static laq_status check_strides_qk(const laq_params* p) {
@@ -217,8 +231,10 @@ laq_status laq_select(const laq_params* p, const float* scores, int32_t* idx,
   d.Ls = d.L - d.R;
   d.Kb = d.B - d.R;
   d.U = (int64_t)d.NL * d.Bt * d.Hkv;
+  laq_status st = derive_seq_lens(p, &d.sl);
+  if (st != LAQ_OK) return st;
   int launches = 0;
-  laq_status st = select_launch(d, scores, idx, (cudaStream_t)cuda_stream, &launches);
+  st = select_launch(d, scores, idx, (cudaStream_t)cuda_stream, &launches);
   g_last_launches = launches;
   return st;
 }

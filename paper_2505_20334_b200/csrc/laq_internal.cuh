@@ -8,6 +8,16 @@
 
 namespace laq {
 
+// Per-prompt lengths, passed to the kernels by value (n = 0: every prompt holds L positions).
+struct SeqLens {
+  int n;
+  int len[LAQ_MAX_RAGGED_BATCH];
+};
+// Length of the prompt of batch item b.
+__host__ __device__ __forceinline__ int unit_len(const SeqLens& sl, int b, int L) {
+  return sl.n > 0 ? sl.len[b] : L;
+}
+
 // Problem sizes derived from laq_params (notation of laq.h).
 struct Dims {
   int NL, Bt, Hq, Hkv, G, D, L, W, R, kpool, B;
@@ -18,7 +28,8 @@ struct Dims {
   int Ls, Kb;   // scored positions, selected slots
   int64_t U;    // units
   float scale;  // softmax scale
-  int tiles_per_task, sched_lag_units;  // caller's scheduling knobs (0 = automatic)
+  int tiles_per_task, sched_lag_tasks;  // caller's scheduling knobs (0 = automatic)
+  SeqLens sl;   // per-prompt lengths (n = 0: uniform)
 };
 
 // Workspace layout (all offsets in bytes from the 256-byte aligned base).

@@ -47,13 +47,14 @@ __device__ __forceinline__ uint4 ld_stream16(const void* p) {
 // total of key i in lane i: one coalesced 128-byte store per warp and round.
 __global__ void __launch_bounds__(kRawThreads) score_raw_d128_kernel(
     const __nv_bfloat16* __restrict__ k, const float* __restrict__ qsum, float* __restrict__ colsum,
-    int Bt, int Hkv, int L, int L_pad, float scale, int64_t s_layer, int64_t s_batch,
-    int64_t s_head, int64_t s_pos) {
+    int Bt, int Hkv, int L_alloc, int L_pad, float scale, int64_t s_layer, int64_t s_batch,
+    int64_t s_head, int64_t s_pos, const __grid_constant__ SeqLens sl) {
   const int64_t u = blockIdx.x;
   const int h = (int)(u % Hkv);
   const int64_t lb = u / Hkv;
   const int b = (int)(lb % Bt);
   const int64_t layer = lb / Bt;
+  const int L = unit_len(sl, b, L_alloc);  // this prompt's own length
   const __nv_bfloat16* ku = k + layer * s_layer + b * s_batch + h * s_head;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int sub = lane & 15, half = lane >> 4;
@@ -112,15 +113,16 @@ __global__ void __launch_bounds__(kRawThreads) score_raw_d128_kernel(
 // Any head_dim that is a multiple of 8 (up to 256): one thread per key, qsum in shared memory.
 __global__ void score_raw_any_kernel(const __nv_bfloat16* __restrict__ k,
                                      const float* __restrict__ qsum, float* __restrict__ colsum,
-                                     int Bt, int Hkv, int D, int L, int L_pad, float scale,
+                                     int Bt, int Hkv, int D, int L_alloc, int L_pad, float scale,
                                      int64_t s_layer, int64_t s_batch, int64_t s_head,
-                                     int64_t s_pos) {
+                                     int64_t s_pos, const __grid_constant__ SeqLens sl) {
   __shared__ float s_q[256];
   const int64_t u = blockIdx.x;
   const int h = (int)(u % Hkv);
   const int64_t lb = u / Hkv;
   const int b = (int)(lb % Bt);
   const int64_t layer = lb / Bt;
+  const int L = unit_len(sl, b, L_alloc);
   for (int d = threadIdx.x; d < D; d += blockDim.x) s_q[d] = qsum[u * D + d];
   __syncthreads();
   const int j = blockIdx.y * blockDim.x + threadIdx.x;
@@ -158,13 +160,13 @@ laq_status score_raw_launch(const laq_params& p, const Dims& d, const Workspace&
     if (chunks > 65535) return LAQ_ERR_UNSUPPORTED;
     score_raw_d128_kernel<<<dim3((unsigned)d.U, chunks), kRawThreads, 0, stream>>>(
         kb, qsum, colsum, d.Bt, d.Hkv, d.L, w.L_pad, d.scale, p.k_stride_layer, p.k_stride_batch,
-        p.k_stride_head, p.k_stride_pos);
+        p.k_stride_head, p.k_stride_pos, d.sl);
   } else {
     const unsigned chunks = (unsigned)((d.L + 255) / 256);
     if (chunks > 65535) return LAQ_ERR_UNSUPPORTED;
     score_raw_any_kernel<<<dim3((unsigned)d.U, chunks), 256, 0, stream>>>(
         kb, qsum, colsum, d.Bt, d.Hkv, d.D, d.L, w.L_pad, d.scale, p.k_stride_layer,
-        p.k_stride_batch, p.k_stride_head, p.k_stride_pos);
+        p.k_stride_batch, p.k_stride_head, p.k_stride_pos, d.sl);
   }
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;

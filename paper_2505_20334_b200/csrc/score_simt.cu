@@ -24,6 +24,7 @@ struct SimtArgs {
   float2* part;
   float* row_off;
   float* colsum;
+  SeqLens sl;  // per-prompt lengths; a.L is the allocated length
 };
 
 __device__ __forceinline__ void unit_coords(const SimtArgs& a, int64_t u, int& layer, int& b,
@@ -77,12 +78,13 @@ __global__ void simt_stats_kernel(SimtArgs a) {
   unit_coords(a, u, layer, b, h);
   stage_q(a, u, 0, a.M_pad, sq, qstride4);
   const __nv_bfloat16* kbase = a.k + layer * a.ks_layer + b * a.ks_batch + h * a.ks_head;
+  const int Lu = unit_len(a.sl, b, a.L);  // this prompt's own length
   const int j0 = chunk * a.keys_per_chunk;
-  const int j1 = min(a.L, j0 + a.keys_per_chunk);
+  const int j1 = min(Lu, j0 + a.keys_per_chunk);
   const int r = threadIdx.x;
   // keys this row may see: a causal local query (LAQ++) stops at its own position
   const int qi = r % a.W;
-  const int vis = qi < a.W_local ? a.L - a.W_local + qi + 1 : a.L;
+  const int vis = qi < a.W_local ? Lu - a.W_local + qi + 1 : Lu;
   float m = -1e30f, l = 0.f;
   for (int js = j0; js < j1; js += kStageKeys) {
     const int nk = min(kStageKeys, j1 - js);
@@ -137,11 +139,13 @@ __global__ void simt_colsum_kernel(SimtArgs a) {
   int layer, b, h;
   unit_coords(a, u, layer, b, h);
   const __nv_bfloat16* kbase = a.k + layer * a.ks_layer + b * a.ks_batch + h * a.ks_head;
+  const int Lu = unit_len(a.sl, b, a.L);
   const int j0 = blockIdx.y * kColTile;
+  if (j0 >= Lu) return;  // block-uniform
   for (int i = threadIdx.x; i < kColTile * dv; i += blockDim.x) {
     const int j = j0 + i / dv;
     uint4 val = make_uint4(0, 0, 0, 0);
-    if (j < a.L) val = reinterpret_cast<const uint4*>(kbase + (int64_t)j * a.ks_pos)[i % dv];
+    if (j < Lu) val = reinterpret_cast<const uint4*>(kbase + (int64_t)j * a.ks_pos)[i % dv];
     sk[(i / dv) * stride4 + (i % dv)] = val;
   }
   float sum = 0.f;
@@ -160,7 +164,7 @@ __global__ void simt_colsum_kernel(SimtArgs a) {
     }
   }
   const int j = j0 + threadIdx.x;
-  if (j < a.L) a.colsum[u * a.L_pad + j] = sum;
+  if (j < Lu) a.colsum[u * a.L_pad + j] = sum;
 }
 
 }  // namespace
@@ -182,6 +186,7 @@ laq_status score_simt_launch(const laq_params& p, const Dims& d, const Workspace
   a.part = (float2*)(ws + w.off_part);
   a.row_off = (float*)(ws + w.off_rowoff);
   a.colsum = (float*)(ws + w.off_colsum);
+  a.sl = d.sl;
   if (d.U > 0x7fffffff || w.L_pad / kColTile > 65535) return LAQ_ERR_UNSUPPORTED;
   const int dv = d.D / 8;
   const size_t smem_stats = ((size_t)w.M_pad * (dv + 1) + (size_t)kStageKeys * dv) * sizeof(uint4);

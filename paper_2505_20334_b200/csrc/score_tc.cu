@@ -8,9 +8,9 @@
 //   sweep 2 (column sums) S^T = K Q^T : rows = keys on the TMEM lanes, so every thread owns one key
 //                         and sums 2^(t[r][j] - b_r) over the rows r, b_r = m_r + log2(l_r).
 // Both sweeps read the same K tile layout (TMA, 128-byte swizzle) and differ only in which operand
-// the tile is. Tickets are ordered so that sweep 2 of a unit is handed out only after sweep 1 of
-// that unit (and of a few later units) has been handed out, so the second sweep re-reads K while
-// it is still resident in L2. A sweep-2 task needs the unit's row statistics, i.e. the partial
+// the tile is. Tickets alternate between the two sweeps, the second trailing the first by a fixed
+// number of tasks: far enough that a unit's statistics are final when its second sweep starts,
+// near enough that the second sweep re-reads K while it is still resident in L2. A sweep-2 task needs the unit's row statistics, i.e. the partial
 // statistics of every sweep-1 task of the unit; those tasks have smaller tickets, which running
 // CTAs already hold, so the order is deadlock-free for any grid size. Every wait is bounded.
 //
@@ -51,7 +51,7 @@ constexpr int kTaskSlots = 4;
 constexpr int kMaxSlots = 4;  // K stages in shared memory = TMEM accumulator buffers
 constexpr int kStatSlots = 2;
 constexpr uint32_t kKStageBytes = TILE_KEYS * 128 * 2;  // 128 keys x 128 dims x bf16
-constexpr uint32_t kCtlBytes = 22528;
+constexpr uint32_t kCtlBytes = 24576;
 constexpr long long kTimeoutCycles = 4000000000LL;  // ~2 s: every device-side wait gives up after this
 constexpr float kLog2e = 1.4426950408889634f;
 // two MMA lanes, statistics-out warp, statistics-in warps, softmax warps
@@ -60,7 +60,9 @@ constexpr int kTaskConsumers = 3 + kStatInWarps + kSoftmaxWarps;
 struct TcArgs {
   int64_t U;
   int Bt, Hkv, G, W, W_local, L, M, M_pad, n_part, L_pad, n_tiles;
-  int tiles_per_task, tasks_per_unit, lag_units;
+  int tiles_per_task, tasks_per_unit;
+  int lag_tasks;        // tasks the second sweep trails the first by
+  int tasks_per_layer;  // per-prompt lengths: sweep-1 tasks of one layer (all prompts and KV heads)
   uint32_t total_tickets;
   float scale_log2;
   int32_t* hdr;
@@ -71,6 +73,7 @@ struct TcArgs {
   int n_slots;     // K stages = accumulator buffers (4, or 2 when a buffer takes 256 columns)
   int slot_shift;  // log2(n_slots)
   int tb_cols;     // TMEM columns per accumulator buffer (128 or 256)
+  SeqLens sl;      // per-prompt lengths (n = 0: every prompt holds L positions)
 };
 
 struct Task {
@@ -79,6 +82,7 @@ struct Task {
   int tile0, n_tiles;
   int chunk;
   int layer, b, h;
+  int L;  // length of this unit's prompt (<= the allocated L)
 };
 
 // Control block at the start of dynamic shared memory.
@@ -98,10 +102,14 @@ struct Ctl {
   uint32_t pad_[2];
   // per finished sweep-1 task: (shift, sum) of every row as seen by each softmax warpgroup
   float2 stat[kStatSlots][kSoftmaxWgs][256];
-  // per sweep-2 task: -b_r of every row (rows beyond M hold -1e30 so that they add nothing)
-  float nboff[kStatSlots][256];
+  // per sweep-2 task: -b_r of every row (rows beyond M hold -1e30 so that they add nothing);
+  // read 16 bytes at a time
+  alignas(16) float nboff[kStatSlots][256];
   // the same offsets prepared for the clamped FMA-pipe exponential: 1/2 - b_r/252
-  float nbsat[kStatSlots][256];
+  alignas(16) float nbsat[kStatSlots][256];
+  // per-prompt lengths: task_prefix[b] = sweep-1 tasks of one layer that belong to prompts < b
+  // (written and read by the producer lane only)
+  int task_prefix[LAQ_MAX_RAGGED_BATCH + 1];
 };
 static_assert(sizeof(Ctl) <= kCtlBytes, "control block too large");
 
@@ -264,34 +272,64 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
   return v;
 }
 
-// Ticket -> task. Order: unit steps i = 0 .. U+lag-1; step i hands out the sweep-1 tasks of unit i
-// (if i < U) and then the sweep-2 tasks of unit i-lag (if i >= lag).
-__device__ __forceinline__ void decode_ticket(const TcArgs& a, uint32_t t, Task& task) {
-  const uint32_t tpu = (uint32_t)a.tasks_per_unit;
-  const uint32_t lag = (uint32_t)a.lag_units;
-  const uint32_t head = lag * tpu;
-  const uint32_t mid = ((uint32_t)a.U - lag) * 2u * tpu;
+// Sweep-1 tasks of a unit whose prompt holds L_unit positions, i.e. the partial statistics it
+// delivers.
+__device__ __forceinline__ int unit_partials(const TcArgs& a, int L_unit) {
+  const int tiles = (L_unit + TILE_KEYS - 1) / TILE_KEYS;
+  return (tiles + a.tiles_per_task - 1) / a.tiles_per_task;
+}
+
+// Ticket -> task. The tasks of one sweep form a stream (layer, prompt, KV head, chunk in row-major
+// order; with per-prompt lengths a unit has as many tasks as its prompt has chunks) of N tasks.
+// The tickets interleave the two streams one task at a time with sweep 2 trailing by lag_tasks:
+// S1[0..lag), then S1[lag+i], S2[i] in turn, then the rest of S2. lag_tasks is at least the
+// largest number of tasks of a unit, so every sweep-1 task of a unit has a smaller ticket than
+// any of its sweep-2 tasks.
+__device__ __forceinline__ void decode_stream(const TcArgs& a, const int* prefix, uint32_t t,
+                                              int& sweep, uint32_t& unit, uint32_t& chunk) {
+  const uint32_t N = a.total_tickets / 2u, lag = (uint32_t)a.lag_tasks;
+  uint32_t i;  // index in the sweep's stream
+  if (t < lag) {
+    sweep = 0; i = t;
+  } else if (t < lag + 2u * (N - lag)) {
+    const uint32_t x = t - lag;
+    if ((x & 1u) == 0) { sweep = 0; i = lag + x / 2u; }
+    else               { sweep = 1; i = x / 2u; }
+  } else {
+    sweep = 1; i = N - lag + (t - lag - 2u * (N - lag));
+  }
+  if (a.sl.n == 0) {  // every prompt of the same length
+    unit = i / (uint32_t)a.tasks_per_unit;
+    chunk = i % (uint32_t)a.tasks_per_unit;
+    return;
+  }
+  const uint32_t layer = i / (uint32_t)a.tasks_per_layer;
+  int r = (int)(i % (uint32_t)a.tasks_per_layer);
+  int lo = 0, hi = a.Bt;  // the prompt b with prefix[b] <= r < prefix[b+1]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (prefix[mid] <= r) lo = mid; else hi = mid;
+  }
+  r -= prefix[lo];
+  const int np = unit_partials(a, a.sl.len[lo]);
+  unit = (layer * (uint32_t)a.Bt + (uint32_t)lo) * (uint32_t)a.Hkv + (uint32_t)(r / np);
+  chunk = (uint32_t)(r % np);
+}
+
+__device__ __forceinline__ void decode_ticket(const TcArgs& a, const int* prefix, uint32_t t,
+                                              Task& task) {
   uint32_t unit, chunk;
   int sweep;
-  if (t < head) {
-    sweep = 0; unit = t / tpu; chunk = t % tpu;
-  } else if (t < head + mid) {
-    const uint32_t x = t - head;
-    const uint32_t step = lag + x / (2u * tpu), w = x % (2u * tpu);
-    if (w < tpu) { sweep = 0; unit = step; chunk = w; }
-    else         { sweep = 1; unit = step - lag; chunk = w - tpu; }
-  } else {
-    const uint32_t x = t - head - mid;
-    sweep = 1; unit = (uint32_t)a.U - lag + x / tpu; chunk = x % tpu;
-  }
+  decode_stream(a, prefix, t, sweep, unit, chunk);
   task.sweep = sweep;
   task.unit = (int)unit;
   task.chunk = (int)chunk;
-  task.tile0 = (int)chunk * a.tiles_per_task;
-  task.n_tiles = min(a.tiles_per_task, a.n_tiles - task.tile0);
   task.h = (int)(unit % (uint32_t)a.Hkv);
   task.b = (int)((unit / (uint32_t)a.Hkv) % (uint32_t)a.Bt);
   task.layer = (int)(unit / ((uint32_t)a.Hkv * (uint32_t)a.Bt));
+  task.L = unit_len(a.sl, task.b, a.L);
+  task.tile0 = (int)chunk * a.tiles_per_task;
+  task.n_tiles = min(a.tiles_per_task, (task.L + TILE_KEYS - 1) / TILE_KEYS - task.tile0);
 }
 
 // Every consumer warp reads the task ring the same way.
@@ -362,7 +400,7 @@ __device__ __forceinline__ void stats_cols64(uint32_t taddr, float c, float& m, 
 // ------------------------------------------------------------------ the kernel
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
-                const __grid_constant__ CUtensorMap tmap_k, const TcArgs a) {
+                const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ TcArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   Ctl* ctl = reinterpret_cast<Ctl*>(smem_raw);
   const uint32_t smem_base = smem_u32(smem_raw);
@@ -426,7 +464,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       uint32_t kcount = 0, qcount = 0, tcount = 0;
       const uint64_t pol_keep = l2_policy_evict_last(), pol_drop = l2_policy_evict_first();
       unsigned int* ticket_ctr = reinterpret_cast<unsigned int*>(&a.hdr[HDR_TICKET]);
-      const Task stop = {-1, 0, 0, 0, 0, 0, 0, 0};
+      const Task stop = {-1, 0, 0, 0, 0, 0, 0, 0, 0};
       // Asks L2 for tiles [first, first+count) of a sweep-1 task ahead of the loads into shared
       // memory, so that the DRAM latency is not paid inside the shared-memory ring.
       auto prefetch_tiles = [&](const Task& t, int first, int count) {
@@ -438,10 +476,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
           tma_prefetch_5d(&tmap_k, 64, key0, t.h, t.b, t.layer, pol_keep);
         }
       };
+      int* prefix = ctl->task_prefix;
+      if (a.sl.n > 0) {
+        int acc = 0;
+        for (int b = 0; b < a.Bt; ++b) {
+          prefix[b] = acc;
+          acc += a.Hkv * unit_partials(a, a.sl.len[b]);
+        }
+        prefix[a.Bt] = acc;
+      }
       Task task = stop;
       {
         const uint32_t t0 = atomicAdd(ticket_ctr, 1u);
-        if (t0 < a.total_tickets) decode_ticket(a, t0, task);
+        if (t0 < a.total_tickets) decode_ticket(a, prefix, t0, task);
       }
       if (LAQ_PREFETCH_TILES > 0) prefetch_tiles(task, 0, LAQ_PREFETCH_TILES);
       bool ok = true;
@@ -494,13 +541,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
             } else {
               if (!next_known) {
                 next_known = true;
-                if (next_ticket < a.total_tickets) decode_ticket(a, next_ticket, next);
+                if (next_ticket < a.total_tickets) decode_ticket(a, prefix, next_ticket, next);
               }
               prefetch_tiles(next, ahead - task.n_tiles, 1);
             }
           }
         }
-        if (!next_known && next_ticket < a.total_tickets) decode_ticket(a, next_ticket, next);
+        if (!next_known && next_ticket < a.total_tickets) decode_ticket(a, prefix, next_ticket, next);
         task = next;
       }
       if (ctl->abort) {
@@ -606,14 +653,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       if (task.sweep != 1) continue;
       const uint32_t s = sc % kStatSlots;
       if (!mbar_wait(a, ctl, smem_u32(&ctl->boff_empty[s]), ((sc / kStatSlots) & 1u) ^ 1u, 41)) break;
-      // every sweep-1 task of the unit must have delivered its partial
+      // every sweep-1 task of the unit that holds tiles must have delivered its partial
+      const int n_partials = unit_partials(a, task.L);
       int ready = 1;
       if (lane == 0) {
         const int32_t* ctr = &a.cnt[task.unit];
-        if (ld_acquire(ctr) < a.tasks_per_unit) {
+        if (ld_acquire(ctr) < n_partials) {
           const long long t0 = clock64();
           uint32_t spins = 0;
-          while (ld_acquire(ctr) < a.tasks_per_unit) {
+          while (ld_acquire(ctr) < n_partials) {
             if ((++spins & 15u) == 0) {
               if (ctl->abort) { ready = 0; break; }
               if (clock64() - t0 > kTimeoutCycles) { record_timeout(a, ctl, 42); ready = 0; break; }
@@ -631,21 +679,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
           float m = -1e30f, l = 0.f;
           const float2* pp = src + row;
           int c0 = 0;
-          for (; c0 + 32 <= a.tasks_per_unit; c0 += 32) {
+          for (; c0 + 32 <= n_partials; c0 += 32) {
             float2 pr[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) pr[i] = __ldcg(pp + (int64_t)(c0 + i) * a.M_pad);
 #pragma unroll
             for (int i = 0; i < 32; ++i) merge_stat(m, l, pr[i]);
           }
-          for (; c0 + 8 <= a.tasks_per_unit; c0 += 8) {
+          for (; c0 + 8 <= n_partials; c0 += 8) {
             float2 pr[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) pr[i] = __ldcg(pp + (int64_t)(c0 + i) * a.M_pad);
 #pragma unroll
             for (int i = 0; i < 8; ++i) merge_stat(m, l, pr[i]);
           }
-          for (; c0 < a.tasks_per_unit; ++c0) merge_stat(m, l, __ldcg(pp + (int64_t)c0 * a.M_pad));
+          for (; c0 < n_partials; ++c0) merge_stat(m, l, __ldcg(pp + (int64_t)c0 * a.M_pad));
           nb = -(m + log2f(l));
         }
         ctl->nboff[s][row] = nb;
@@ -669,11 +717,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
     const int ch_lo = half == 0 ? 0 : (n_chunks2 + 1) / 2;
     const int ch_hi = half == 0 ? (n_chunks2 + 1) / 2 : n_chunks2;
     const uint32_t col0 = 64u * (uint32_t)half;  // sweep 1: this warpgroup's 64 key columns
-    // keys [0, vis) are visible to this thread's query rows: all L for a lookahead query, the
-    // positions up to its own for a local query (query i of a head sits at L - W_local + i)
-    const int qi0 = row_in_wg % a.W, qi1 = (128 + row_in_wg) % a.W;
-    const int vis0 = qi0 < a.W_local ? a.L - a.W_local + qi0 + 1 : a.L;
-    const int vis1 = qi1 < a.W_local ? a.L - a.W_local + qi1 + 1 : a.L;
+    const int qi0 = row_in_wg % a.W, qi1 = (128 + row_in_wg) % a.W;  // query index inside its head
     // Tiles are numbered through all tasks of this CTA; pair p owns tiles p, p + 2, ... A parity
     // wait is sound because the previous use of a slot (tile t - n_slots) is never later than the
     // pair's previous tile (t - 2).
@@ -684,6 +728,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       if (!next_task(a, ctl, tk, lane, false, 20, task)) break;
       if (task.sweep < 0) break;
       const int64_t u = task.unit;
+      // keys [0, vis) of this unit's Lu are visible to this thread's query rows: all of them for a
+      // lookahead query, the positions up to its own for a local query (query i of a head sits at
+      // Lu - W_local + i)
+      const int Lu = task.L;
+      const int vis0 = qi0 < a.W_local ? Lu - a.W_local + qi0 + 1 : Lu;
+      const int vis1 = qi1 < a.W_local ? Lu - a.W_local + qi1 + 1 : Lu;
       float m0 = -1e30f, l0 = 0.f, m1 = -1e30f, l1 = 0.f;
       const float* nboff = nullptr;
       const float* nbsat = nullptr;
@@ -708,10 +758,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         const uint32_t empty_bar = smem_u32(&ctl->tmem_empty[s]);
         float v[32];
         if (task.sweep == 0) {
-          const int valid = min(TILE_KEYS, a.L - key0);
+          const int valid = min(TILE_KEYS, Lu - key0);
           // row blocks beyond the unit's rows are skipped (warp-uniform)
           const bool rows0 = quad * 32 < a.M, rows1 = RB == 2 && 128 + quad * 32 < a.M;
-          if (valid == TILE_KEYS && key0 + TILE_KEYS <= a.L - a.W_local) {
+          if (valid == TILE_KEYS && key0 + TILE_KEYS <= Lu - a.W_local) {
             // every column is a real key that every row sees
             if (rows0) stats_cols64(taddr + col0, c, m0, l0, v, !rows1, empty_bar, lane);
             if (rows1) stats_cols64(taddr + 128u + col0, c, m1, l1, v, true, empty_bar, lane);
@@ -749,7 +799,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
             // sum; with at most two addends the result does not depend on the order.
             const float2 s2 = __fadd2_rn(__fadd2_rn(acc[0], acc[1]), __fadd2_rn(acc[2], acc[3]));
             const int key = key0 + row_in_wg;
-            if (key < a.L) red_add(&a.colsum[u * a.L_pad + key], s2.x + s2.y);
+            if (key < Lu) red_add(&a.colsum[u * a.L_pad + key], s2.x + s2.y);
           }
         }
       }
@@ -837,32 +887,49 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   // every chunk must hold at least one tile
   if ((a.tasks_per_unit - 1) * a.tiles_per_task >= a.n_tiles || d.W > 256 || d.G > 256)
     return score_simt_launch(p, d, w, q, k, ws, stream, launches);
-  const uint64_t tickets = 2ull * (uint64_t)d.U * (uint64_t)a.tasks_per_unit;
-  if (tickets >= 0x7fffffffull || d.U >= 0x7fffffff) return LAQ_ERR_UNSUPPORTED;
-  a.total_tickets = (uint32_t)tickets;
+  if (d.U >= 0x7fffffff) return LAQ_ERR_UNSUPPORTED;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
     return LAQ_ERR_CUDA;
-  // Sweep 2 trails sweep 1 by `lag` units. Too short and sweep-2 tasks wait for statistics that
-  // are not final yet; too long and K has left L2 when the second sweep reads it again. Measured
-  // on B200 (8 MiB of K per unit): 48 MiB of K between the sweeps re-reads everything from L2
-  // (9.3 GB of DRAM traffic per 8.6 GB of K), 64 MiB re-reads everything from HBM (15.8 GB); and
-  // about 1.3 tickets per SM is the shortest distance at which sweep 2 rarely waits.
-  int lag = d.sched_lag_units;
-  if (lag <= 0) {
-    const int64_t k_unit_bytes = (int64_t)d.L * d.D * 2;
-    const int by_l2 = (int)((48ll << 20) / (k_unit_bytes > 0 ? k_unit_bytes : 1));
-    const int by_latency = (5 * sms / 4 + 2 * a.tasks_per_unit - 1) / (2 * a.tasks_per_unit);
-    lag = by_l2 > by_latency ? by_l2 : by_latency;
+  // One ticket per task that holds tiles (with per-prompt lengths a short prompt has fewer).
+  int64_t n_stream = (int64_t)d.U * a.tasks_per_unit;
+  a.tasks_per_layer = 0;
+  if (d.sl.n > 0) {
+    int64_t per_layer = 0;
+    for (int b = 0; b < d.Bt; ++b) {
+      const int tiles = (d.sl.len[b] + TILE_KEYS - 1) / TILE_KEYS;
+      per_layer += (int64_t)d.Hkv * ((tiles + a.tiles_per_task - 1) / a.tiles_per_task);
+    }
+    n_stream = per_layer * d.NL;
+    a.tasks_per_layer = (int)per_layer;
   }
-  if ((int64_t)lag > d.U) lag = (int)d.U;
-  a.lag_units = lag;
+  if (2 * n_stream >= 0x7fffffffll) return LAQ_ERR_UNSUPPORTED;
+  a.total_tickets = (uint32_t)(2 * n_stream);
+  // Sweep 2 trails sweep 1 by lag_tasks tasks. Too short and sweep-2 tasks wait for statistics
+  // that are not final yet; too long and K has left L2 when the second sweep reads it again.
+  // Measured on B200: the best distance is as much K as L2 still returns (about 52 MiB: 104-116
+  // tasks of 16 tiles at L = 32768, 208 tasks of 8 tiles at L = 16384), but never less than the
+  // tasks of one unit plus the tasks that half the SMs start while one task runs and its
+  // statistics travel (about 4 us); a 128-key tile takes 0.7-1.6 us per sweep depending on M.
+  int64_t lag_tasks = d.sched_lag_tasks;
+  if (lag_tasks <= 0) {
+    const int64_t task_bytes = (int64_t)a.tiles_per_task * TILE_KEYS * d.D * 2;
+    const int64_t by_l2 = (52ll << 20) / task_bytes;
+    const double tile_us = w.M_pad <= 64 ? 0.7 : (w.M_pad <= 128 ? 0.8 : 1.6);
+    const int64_t by_latency =
+        a.tasks_per_unit + (int64_t)(0.5 * sms * (1.0 + 4.0 / (a.tiles_per_task * tile_us)) + 0.999);
+    lag_tasks = by_l2 > by_latency ? by_l2 : by_latency;
+  }
+  if (lag_tasks < a.tasks_per_unit) lag_tasks = a.tasks_per_unit;
+  if (lag_tasks > n_stream) lag_tasks = n_stream;
+  a.lag_tasks = (int)lag_tasks;
   a.scale_log2 = d.scale * kLog2e;
   a.hdr = (int32_t*)(ws + w.off_hdr);
   a.cnt = (int32_t*)(ws + w.off_cnt);
   a.part = (float2*)(ws + w.off_part);
   a.colsum = (float*)(ws + w.off_colsum);
+  a.sl = d.sl;
   const bool wide = d.M > 128;
   a.q_rows = wide ? 256 : 128;
   a.n_slots = wide ? 2 : 4;

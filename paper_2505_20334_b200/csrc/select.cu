@@ -9,6 +9,16 @@ namespace {
 constexpr int kSelThreads = 1024;
 constexpr int kSelWarps = kSelThreads / 32;
 
+// Geometry shared by the kernels below. Ls_full = L - R is the row length of the score tensor;
+// a unit whose prompt is shorter (per-prompt lengths) scores only its first Lb - R positions.
+struct SelGeom {
+  int Ls_full, Kb, R, B, Bt, Hkv;
+  SeqLens sl;
+};
+__device__ __forceinline__ int unit_scored(const SelGeom& g, int64_t u) {
+  return unit_len(g.sl, (int)((u / g.Hkv) % g.Bt), g.Ls_full + g.R) - g.R;
+}
+
 // Average pooling: p_j = (1/k) * sum_{|t| <= k/2, 0 <= j+t < Ls} c_{j+t} (zero padding, divisor
 // always k). Maximum pooling: the largest c_{j+t} over the same window positions that exist.
 // One position near an edge of [0, Ls), or any position when the window is not unrolled.
@@ -31,11 +41,14 @@ __device__ __forceinline__ float pool_at(const float* c, int j, int h, int Ls, f
 }
 
 __global__ void pool_kernel(const float* __restrict__ colsum, int L_pad, float* __restrict__ pooled,
-                            int Ls, int kpool, float inv_k, int pool_max) {
-  const int64_t u = blockIdx.y;
+                            int kpool, float inv_k, int pool_max, int64_t u0,
+                            const __grid_constant__ SelGeom g) {
+  const int64_t u = u0 + blockIdx.y;
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= Ls) return;
-  pooled[u * Ls + j] = pool_at(colsum + u * L_pad, j, kpool / 2, Ls, inv_k, pool_max);
+  if (j >= g.Ls_full) return;
+  const int Ls = unit_scored(g, u);
+  pooled[u * g.Ls_full + j] =
+      j < Ls ? pool_at(colsum + u * L_pad, j, kpool / 2, Ls, inv_k, pool_max) : 0.f;
 }
 
 // Order-preserving map from fp32 bits to uint32 (larger float <=> larger key).
@@ -146,10 +159,10 @@ __device__ __forceinline__ void select_unit(const float* p, int32_t* out, int Ls
 
 // Step 5 alone: scores of unit blockIdx.x in global memory.
 __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __restrict__ pooled,
-                                                             int32_t* __restrict__ idx, int Ls,
-                                                             int Kb, int R, int B) {
+                                                             int32_t* __restrict__ idx,
+                                                             const __grid_constant__ SelGeom g) {
   const int64_t u = blockIdx.x;
-  select_unit(pooled + u * (int64_t)Ls, idx + u * (int64_t)B, Ls, Kb, R);
+  select_unit(pooled + u * (int64_t)g.Ls_full, idx + u * (int64_t)g.B, unit_scored(g, u), g.Kb, g.R);
 }
 
 // Steps 4 and 5 in one pass over the column sums: the block pools its unit's scores into shared
@@ -157,20 +170,21 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
 // radix passes never go back to global memory. The pooling arithmetic is that of pool_kernel.
 __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const float* __restrict__ colsum,
                                                                   int L_pad, float* pooled_out,
-                                                                  int32_t* __restrict__ idx, int Ls,
-                                                                  int Kb, int R, int B, int kpool,
-                                                                  float inv_k, int pool_max) {
+                                                                  int32_t* __restrict__ idx, int kpool,
+                                                                  float inv_k, int pool_max,
+                                                                  const __grid_constant__ SelGeom g) {
   extern __shared__ float s_pooled[];
   const int64_t u = blockIdx.x;
   const float* c = colsum + u * (int64_t)L_pad;
   const int h = kpool / 2;
-  for (int j = threadIdx.x; j < Ls; j += kSelThreads) {
-    const float pj = pool_at(c, j, h, Ls, inv_k, pool_max);
-    s_pooled[j] = pj;
-    if (pooled_out) pooled_out[u * (int64_t)Ls + j] = pj;
+  const int Ls = unit_scored(g, u);
+  for (int j = threadIdx.x; j < g.Ls_full; j += kSelThreads) {
+    const float pj = j < Ls ? pool_at(c, j, h, Ls, inv_k, pool_max) : 0.f;
+    if (j < Ls) s_pooled[j] = pj;
+    if (pooled_out) pooled_out[u * (int64_t)g.Ls_full + j] = pj;
   }
   __syncthreads();
-  select_unit(s_pooled, idx + u * (int64_t)B, Ls, Kb, R);
+  select_unit(s_pooled, idx + u * (int64_t)g.B, Ls, g.Kb, g.R);
 }
 
 // Steps 4 and 5 for units of at most kRegItems * 1024 scored positions, with the unit's pooled
@@ -206,13 +220,14 @@ __device__ __forceinline__ void transpose32(uint32_t (&a)[32]) {
 // kPoolStatic > 0 fixes the pooling kernel at compile time (unrolled taps); 0 takes it from `kpool`.
 template <int kPoolStatic>
 __global__ void __launch_bounds__(kSelThreads) pool_select_reg_kernel(
-    const float* __restrict__ colsum, int L_pad, float* pooled_out, int32_t* __restrict__ idx, int Ls,
-    int Kb, int R, int B, int kpool, float inv_k, int pool_max) {
+    const float* __restrict__ colsum, int L_pad, float* pooled_out, int32_t* __restrict__ idx,
+    int kpool, float inv_k, int pool_max, const __grid_constant__ SelGeom g) {
   __shared__ uint32_t s_cnt[2][kSelWarps];
   __shared__ uint32_t s_gt[kSelWarps], s_eq[kSelWarps];
   const int64_t u = blockIdx.x;
   const float* c = colsum + u * (int64_t)L_pad;
-  int32_t* out = idx + u * (int64_t)B;
+  const int Ls = unit_scored(g, u), Kb = g.Kb, R = g.R;
+  int32_t* out = idx + u * (int64_t)g.B;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int base = warp * (kRegItems * 32) + lane;
   const int h = (kPoolStatic > 0 ? kPoolStatic : kpool) / 2;
@@ -240,9 +255,11 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_reg_kernel(
       } else {
         pj = pool_at(c, j, h, Ls, inv_k, pool_max);
       }
-      if (pooled_out) pooled_out[u * (int64_t)Ls + j] = pj;
+      if (pooled_out) pooled_out[u * (int64_t)g.Ls_full + j] = pj;
       key = order_key(pj);
       alive |= 1u << it;
+    } else if (pooled_out && j < g.Ls_full) {
+      pooled_out[u * (int64_t)g.Ls_full + j] = 0.f;  // beyond a shorter prompt's scored positions
     }
     w[it] = key;
   }
@@ -303,20 +320,21 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_reg_kernel(
 
 }  // namespace
 
+static SelGeom sel_geom(const Dims& d) {
+  SelGeom g;
+  g.Ls_full = d.Ls; g.Kb = d.Kb; g.R = d.R; g.B = d.B; g.Bt = d.Bt; g.Hkv = d.Hkv;
+  g.sl = d.sl;
+  return g;
+}
+
 laq_status pool_launch(const Dims& d, const float* colsum, int L_pad, float* pooled,
                        cudaStream_t stream, int* launches) {
-  if (d.U > 65535) {
-    // grid.y limit: launch in slabs of units
-    for (int64_t u0 = 0; u0 < d.U; u0 += 65535) {
-      const unsigned nu = (unsigned)((d.U - u0 < 65535) ? d.U - u0 : 65535);
-      pool_kernel<<<dim3((d.Ls + 255) / 256, nu), 256, 0, stream>>>(
-          colsum + u0 * L_pad, L_pad, pooled + u0 * d.Ls, d.Ls, d.kpool, 1.0f / (float)d.kpool,
-          d.pool_max);
-      *launches += 1;
-    }
-  } else {
-    pool_kernel<<<dim3((d.Ls + 255) / 256, (unsigned)d.U), 256, 0, stream>>>(
-        colsum, L_pad, pooled, d.Ls, d.kpool, 1.0f / (float)d.kpool, d.pool_max);
+  const SelGeom g = sel_geom(d);
+  // grid.y limit: launch in slabs of units
+  for (int64_t u0 = 0; u0 < d.U; u0 += 65535) {
+    const unsigned nu = (unsigned)((d.U - u0 < 65535) ? d.U - u0 : 65535);
+    pool_kernel<<<dim3((d.Ls + 255) / 256, nu), 256, 0, stream>>>(
+        colsum, L_pad, pooled, d.kpool, 1.0f / (float)d.kpool, d.pool_max, u0, g);
     *launches += 1;
   }
   return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;
@@ -325,7 +343,7 @@ laq_status pool_launch(const Dims& d, const float* colsum, int L_pad, float* poo
 laq_status select_launch(const Dims& d, const float* pooled, int32_t* idx, cudaStream_t stream,
                          int* launches) {
   if (d.U > 0x7fffffff) return LAQ_ERR_UNSUPPORTED;
-  select_kernel<<<(unsigned)d.U, kSelThreads, 0, stream>>>(pooled, idx, d.Ls, d.Kb, d.R, d.B);
+  select_kernel<<<(unsigned)d.U, kSelThreads, 0, stream>>>(pooled, idx, sel_geom(d));
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;
 }
@@ -334,13 +352,13 @@ laq_status pool_select_launch(const Dims& d, const float* colsum, int L_pad, flo
                               int32_t* idx, cudaStream_t stream, int* launches, bool* done) {
   *done = false;
   if (d.U > 0x7fffffff) return LAQ_OK;
+  const SelGeom g = sel_geom(d);
   if (d.Ls <= kRegItems * kSelThreads) {
     const float inv_k = 1.0f / (float)d.kpool;
     const unsigned grid = (unsigned)d.U;
 #define LAQ_LAUNCH_POOL_SELECT(KP)                                                         \
   pool_select_reg_kernel<KP><<<grid, kSelThreads, 0, stream>>>(colsum, L_pad, pooled_out, idx, \
-                                                               d.Ls, d.Kb, d.R, d.B, d.kpool, inv_k, \
-                                                               d.pool_max)
+                                                               d.kpool, inv_k, d.pool_max, g)
     switch (d.kpool) {
       case 1: LAQ_LAUNCH_POOL_SELECT(1); break;
       case 3: LAQ_LAUNCH_POOL_SELECT(3); break;
@@ -359,8 +377,7 @@ laq_status pool_select_launch(const Dims& d, const float* colsum, int L_pad, flo
                            (int)smem) != cudaSuccess)
     return LAQ_ERR_CUDA;
   pool_select_kernel<<<(unsigned)d.U, kSelThreads, smem, stream>>>(
-      colsum, L_pad, pooled_out, idx, d.Ls, d.Kb, d.R, d.B, d.kpool, 1.0f / (float)d.kpool,
-      d.pool_max);
+      colsum, L_pad, pooled_out, idx, d.kpool, 1.0f / (float)d.kpool, d.pool_max, g);
   *launches += 1;
   *done = true;
   return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;

@@ -33,7 +33,7 @@ def test_header_symbols_are_exported(binding):
 
 
 def test_struct_layout_and_version(binding):
-    assert ctypes.sizeof(binding.LaqParams) == 16 * 4 + 16 * 8
+    assert ctypes.sizeof(binding.LaqParams) == 16 * 4 + 16 * 8 + 8
     assert binding.LaqParams.q_stride_layer.offset == 64
     assert binding.laq_version() >= 100
     assert binding.status_string(0) == "ok"
@@ -101,3 +101,24 @@ def test_unsupported_and_pointer_checks(binding):
     assert binding.lib.laq_select(ctypes.byref(p), None, fake, None) == binding.LAQ_ERR_INVALID_ARG
     assert binding.lib.laq_compact(ctypes.byref(p), fake, fake, None, fake, fake, None) == \
         binding.LAQ_ERR_INVALID_ARG
+
+
+def test_seq_lens_are_validated_on_host(binding):
+    p = binding.make_params(1, 3, 8, 2, 128, 1000, 4, 4, 7, 64)
+    base = binding.laq_workspace_bytes(p)
+    p.set_seq_lens([1000, 65, 500])
+    assert binding.laq_workspace_bytes(p) == base          # lengths do not change the workspace
+    for bad in ([1000, 64, 500],      # a prompt no longer than the budget
+                [1001, 500, 500],     # longer than the allocated length
+                [1000, 500, -3]):
+        p.set_seq_lens(bad)
+        assert binding.laq_workspace_bytes(p) == 0
+    with pytest.raises(ValueError):
+        p.set_seq_lens([1000, 500])   # one length per batch item
+    p.set_seq_lens(None)
+    assert binding.laq_workspace_bytes(p) == base
+    big = binding.make_params(1, 513, 8, 2, 128, 1000, 4, 4, 7, 64)
+    big.set_seq_lens([1000] * 513)    # more prompts than LAQ_MAX_RAGGED_BATCH
+    fake = ctypes.c_void_p(4096)
+    assert binding.lib.laq_score(ctypes.byref(big), fake, fake, fake, fake, 1 << 40, None) == \
+        binding.LAQ_ERR_UNSUPPORTED

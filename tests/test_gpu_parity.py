@@ -28,18 +28,20 @@ def rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed, kscale=1.0):
     return q, k, v
 
 
-def run_evict(laq, q, k, v, R, kernel, B, local_window=0, pool_mode=0, score_mode=0):
+def run_evict(laq, q, k, v, R, kernel, B, local_window=0, pool_mode=0, score_mode=0, seq_lens=None):
     out = laq.evict(q.cuda(), k.cuda(), v.cuda(), B, pool_kernel=kernel, keep_tail=R,
                     want_scores=True, local_window=local_window, pool_mode=pool_mode,
-                    score_mode=score_mode)
+                    score_mode=score_mode, seq_lens=seq_lens)
     assert laq.laq_last_device_status(out["params"], out["ws"]) == laq.LAQ_OK
     return out
 
 
-def compare_all_units(laq, q, k, v, R, kernel, B, out=None, local_window=0, pool_mode=0):
+def compare_all_units(laq, q, k, v, R, kernel, B, out=None, local_window=0, pool_mode=0,
+                      seq_lens=None):
     """Full comparison of every unit of a (small) problem against the oracle."""
-    out = out or run_evict(laq, q, k, v, R, kernel, B, local_window, pool_mode)
-    ref = orc.evict(q, k, v, R, kernel, B, local_window=local_window, pool_mode=pool_mode)
+    out = out or run_evict(laq, q, k, v, R, kernel, B, local_window, pool_mode, seq_lens=seq_lens)
+    ref = orc.evict(q, k, v, R, kernel, B, local_window=local_window, pool_mode=pool_mode,
+                    seq_lens=seq_lens)
     NL, Bt, Hkv, L = k.shape[0], k.shape[1], k.shape[2], k.shape[3]
     got_scores = out["scores"].cpu().numpy()
     err = score_rel_err(got_scores, ref["scores"])
@@ -50,11 +52,13 @@ def compare_all_units(laq, q, k, v, R, kernel, B, out=None, local_window=0, pool
     differing = 0
     for n in range(NL):
         for b in range(Bt):
+            Lb = L if seq_lens is None else int(seq_lens[b])   # this prompt's own length
             for h in range(Hkv):
                 differing += check_index_set(got_idx[n, b, h], ref["idx"][n, b, h],
-                                             ref["scores"][n, b, h], L, R, B)
+                                             ref["scores"][n, b, h][:Lb - R], Lb, R, B)
+                assert (got_scores[n, b, h][Lb - R:] == 0).all()
                 # selection is bit-exact on the GPU's own scores (tie-break included)
-                want = orc.select(got_scores[n, b, h], L, R, B, sorted_variant=True)
+                want = orc.select(got_scores[n, b, h][:Lb - R], Lb, R, B, sorted_variant=True)
                 assert (got_idx[n, b, h] == want).all()
                 # compaction is bit-exact given the indices
                 assert (ko[n, b, h] == kb[n, b, h][got_idx[n, b, h]]).all()
@@ -270,6 +274,54 @@ def test_raw_logit_mode_matches_oracle(laq, shape):
                 assert (ko[n, b, h] == kb[n, b, h][got_idx[n, b, h]]).all()
                 assert (vo[n, b, h] == vb[n, b, h][got_idx[n, b, h]]).all()
     assert (got_scores < 0).any() and (got_scores > 0).any()
+
+
+RAGGED_SHAPES = [
+    # NL Bt Hq Hkv D    L     W  W_local k  B    lens
+    (1, 3, 8, 2, 128, 1500, 16, 0, 7, 100, (1500, 333, 901)),    # second chunk of prompt 1 is empty
+    (2, 2, 4, 1, 128, 3000, 32, 16, 5, 200, (2049, 3000)),       # M = 128, LAQ++ window at each prompt's own end
+    (1, 2, 8, 1, 128, 1536, 32, 0, 7, 64, (700, 1536)),          # M = 256
+    (1, 4, 4, 2, 128, 600, 8, 8, 3, 40, (41, 128, 129, 600)),    # shortest legal prompt, tile edges
+    (1, 2, 8, 2, 64, 500, 8, 4, 7, 90, (500, 200)),              # head_dim 64: CUDA-core path
+]
+
+
+@pytest.mark.parametrize("shape", RAGGED_SHAPES, ids=[f"L{s[5]}-M{s[2] // s[3] * s[6]}-D{s[4]}" for s in RAGGED_SHAPES])
+def test_prompts_of_different_lengths_match_oracle(laq, shape):
+    NL, Bt, Hq, Hkv, D, L, W, Wl, kernel, B, lens = shape
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=L + sum(lens), kscale=1.5)
+    # rows beyond a prompt's length may hold anything, NaN included
+    for b, Lb in enumerate(lens):
+        k[:, b, :, Lb:] = float("nan")
+        v[:, b, :, Lb:] = float("nan")
+    err, _ = compare_all_units(laq, q, k, v, W, kernel, B, local_window=Wl, seq_lens=lens)
+    assert err < SCORE_RTOL
+    # the separate entry points take the lengths too
+    qc, kc, vc = q.cuda(), k.cuda(), v.cuda()
+    ref = laq.evict(qc, kc, vc, B, pool_kernel=kernel, keep_tail=W, want_scores=True,
+                    local_window=Wl, seq_lens=lens)
+    p = ref["params"]
+    scores = torch.full_like(ref["scores"], -1.0)
+    idx = torch.zeros_like(ref["idx"])
+    laq.laq_score(p, qc, kc, scores, ref["ws"])
+    laq.laq_select(p, scores, idx)
+    assert torch.equal(scores, ref["scores"]) and torch.equal(idx, ref["idx"])
+    # raw-logit mode on the same ragged batch
+    raw = run_evict(laq, q, k, v, W, 1, B, score_mode=1, seq_lens=lens)
+    want = orc.evict(q, k, v, W, 1, B, score_mode=1, seq_lens=lens)
+    got = raw["scores"].cpu().numpy()
+    assert np.isfinite(got).all()
+    np.testing.assert_allclose(got, want["scores"], rtol=0, atol=2e-5 * np.abs(want["scores"]).max() * 8)
+    for b, Lb in enumerate(lens):
+        assert (got[:, b, :, Lb - W:] == 0).all()
+        assert (raw["idx"][:, b, :, B - W:].cpu().numpy() == np.arange(Lb - W, Lb)).all()
+
+
+def test_seq_lens_argument_checks(laq):
+    q, k, v = rand_inputs(1, 2, 4, 2, 128, 300, 8, seed=5)
+    for bad in ((300, 40), (301, 100), (300,)):     # not longer than the budget / too long / too few
+        with pytest.raises((laq.LaqError, ValueError)):
+            laq.evict(q.cuda(), k.cuda(), v.cuda(), 40, seq_lens=bad)
 
 
 def test_variant_argument_checks(laq):
