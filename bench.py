@@ -32,7 +32,8 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one score_tc_kernel launch on this workload,
 # from the ncu capture summarised under profiles/ (None until one has been taken).
-NCU_TRAFFIC_BYTES = 9.45e9
+NCU_TRAFFIC_BYTES = 9.77e9
+NCU_TRAFFIC_BYTES_RAW = 8.68e9  # the same for score_raw_d128_kernel (--score-mode raw)
 
 
 def parse_args():
@@ -331,9 +332,12 @@ def main():
     score_bytes, gather_bytes = algorithmic_bytes(cfg, B, tokens_per_step / Bt)
     achieved = score_bytes / (score_ms * 1e-3) / 1e9
     raw = args.score_mode == "raw"
+    # the ncu figures were taken on the full headline workload only
+    captured = args.config == 3 and not (args.layers or args.batch or args.prompt_len or lens)
+    traffic = (NCU_TRAFFIC_BYTES_RAW if raw else NCU_TRAFFIC_BYTES) if captured else None
     roofline = {"bound": "hbm", "kernel": "score_raw_d128_kernel" if raw else "score_tc_kernel",
                 "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "traffic": None if raw else NCU_TRAFFIC_BYTES,
+                "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
                 "peak_source": peak_src, "algorithmic_bytes_per_launch": score_bytes,
                 "kernel_ms": score_ms, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
     # The scoring kernel's busiest unit is the MUFU: two base-2 exponentials per (row, key) pair
