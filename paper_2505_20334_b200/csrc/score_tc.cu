@@ -73,6 +73,7 @@ struct TcArgs {
   int n_slots;     // K stages = accumulator buffers (4, or 2 when a buffer takes 256 columns)
   int slot_shift;  // log2(n_slots)
   int tb_cols;     // TMEM columns per accumulator buffer (128 or 256)
+  int dup;         // 1 when M <= 64: sweep 1 holds every query row twice, on lanes r and 64 + r
   SeqLens sl;      // per-prompt lengths (n = 0: every prompt holds L positions)
 };
 
@@ -507,11 +508,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
           const uint32_t qs = qcount & 1u;
           if (!mbar_wait(a, ctl, smem_u32(&ctl->q_empty[qs]), ((qcount >> 1) & 1u) ^ 1u, 3)) break;
           const uint32_t bar = smem_u32(&ctl->q_full[qs]);
-          mbar_expect_tx(bar, (uint32_t)a.M * 256u);
+          mbar_expect_tx(bar, (uint32_t)a.M * 256u * (a.dup ? 2u : 1u));
           const uint32_t dst = q_base + qs * q_stage_bytes;
           tma_load_5d(dst, &tmap_q, bar, 0, 0, task.h * a.G, task.b, task.layer);
           tma_load_5d(dst + (uint32_t)a.q_rows * 128u, &tmap_q, bar, 64, 0, task.h * a.G, task.b,
                       task.layer);
+          if (a.dup) {
+            // a second copy of the rows, 64 rows (8192 bytes: the swizzle pattern repeats) further
+            tma_load_5d(dst + 8192u, &tmap_q, bar, 0, 0, task.h * a.G, task.b, task.layer);
+            tma_load_5d(dst + (uint32_t)a.q_rows * 128u + 8192u, &tmap_q, bar, 64, 0, task.h * a.G,
+                        task.b, task.layer);
+          }
           ++qcount;
         }
         // sweep 1 asks L2 to keep the tile for the second sweep, which then lets it go
@@ -631,6 +638,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         float m = -1e30f, l = 0.f;
 #pragma unroll
         for (int g = 0; g < kSoftmaxWgs; ++g) merge_stat(m, l, ctl->stat[s][g][row]);
+        if (a.dup) {  // the second copy of the row saw the other key columns
+#pragma unroll
+          for (int g = 0; g < kSoftmaxWgs; ++g) merge_stat(m, l, ctl->stat[s][g][64 + row]);
+        }
         dst[row] = make_float2(m, l);
       }
       __threadfence();
@@ -717,7 +728,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
     const int ch_lo = half == 0 ? 0 : (n_chunks2 + 1) / 2;
     const int ch_hi = half == 0 ? (n_chunks2 + 1) / 2 : n_chunks2;
     const uint32_t col0 = 64u * (uint32_t)half;  // sweep 1: this warpgroup's 64 key columns
-    const int qi0 = row_in_wg % a.W, qi1 = (128 + row_in_wg) % a.W;  // query index inside its head
+    // Sweep 1 with M <= 64: lanes 64.. hold a second copy of the rows, so the warps on lanes r and
+    // 64 + r share row r's 64 key columns of this warpgroup (32 each) and all four quadrants of
+    // the SM work; otherwise this thread's rows are row_in_wg and 128 + row_in_wg.
+    const int row_s1 = a.dup ? (quad & 1) * 32 + lane : row_in_wg;
+    const uint32_t col_d = 64u * (uint32_t)half + 32u * (uint32_t)(quad >> 1);  // dup: my 32 columns
+    const int qi0 = row_s1 % a.W, qi1 = (128 + row_in_wg) % a.W;  // query index inside its head
     // Tiles are numbered through all tasks of this CTA; pair p owns tiles p, p + 2, ... A parity
     // wait is sound because the previous use of a slot (tile t - n_slots) is never later than the
     // pair's previous tile (t - 2).
@@ -760,8 +776,25 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         if (task.sweep == 0) {
           const int valid = min(TILE_KEYS, Lu - key0);
           // row blocks beyond the unit's rows are skipped (warp-uniform)
-          const bool rows0 = quad * 32 < a.M, rows1 = RB == 2 && 128 + quad * 32 < a.M;
-          if (valid == TILE_KEYS && key0 + TILE_KEYS <= Lu - a.W_local) {
+          const bool rows0 = (a.dup ? (quad & 1) : quad) * 32 < a.M;
+          const bool rows1 = RB == 2 && 128 + quad * 32 < a.M;
+          if (a.dup) {
+            if (!rows0) {
+              release_buffer(empty_bar, lane);
+            } else if (valid == TILE_KEYS && key0 + TILE_KEYS <= Lu - a.W_local) {
+              tmem_ld32(taddr + col_d, v);
+              tmem_ld_wait(v);
+              release_buffer(empty_bar, lane);
+              stats_chunk<LAQ_POLY_PAIRS_S1>(v, c, m0, l0);
+            } else {
+              const int vq = min(32, valid - (int)col_d);
+              const float2 r =
+                  stats_cols_ragged(taddr + col_d, vq, min(vq, vis0 - key0 - (int)col_d), c, m0, l0);
+              m0 = r.x;
+              l0 = r.y;
+              release_buffer(empty_bar, lane);
+            }
+          } else if (valid == TILE_KEYS && key0 + TILE_KEYS <= Lu - a.W_local) {
             // every column is a real key that every row sees
             if (rows0) stats_cols64(taddr + col0, c, m0, l0, v, !rows1, empty_bar, lane);
             if (rows1) stats_cols64(taddr + 128u + col0, c, m1, l1, v, true, empty_bar, lane);
@@ -935,6 +968,7 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   a.n_slots = wide ? 2 : 4;
   a.slot_shift = wide ? 1 : 2;
   a.tb_cols = wide ? 256 : 128;
+  a.dup = w.M_pad <= 64 ? 1 : 0;
 
   CUtensorMap tmap_q, tmap_k;
   const uint64_t qdims[5] = {128, (uint64_t)d.W, (uint64_t)d.Hq, (uint64_t)d.Bt, (uint64_t)d.NL};
