@@ -324,6 +324,38 @@ def test_seq_lens_argument_checks(laq):
             laq.evict(q.cuda(), k.cuda(), v.cuda(), 40, seq_lens=bad)
 
 
+def _random_case(seed):
+    """A small random problem: geometry, options and per-prompt lengths drawn from a seeded stream."""
+    rng = np.random.default_rng(9000 + seed)
+    D = int(rng.choice([128, 128, 128, 64]))
+    Hkv = int(rng.choice([1, 2, 3]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    W = int(rng.choice([1, 3, 8, 16, 32]))
+    while G * W > 256:
+        W //= 2
+    L = int(rng.integers(60, 2600))
+    Bt = int(rng.choice([1, 2, 3]))
+    NL = int(rng.choice([1, 2]))
+    R = W
+    B = int(rng.integers(R + 1, max(R + 2, min(L // 2, 300))))
+    kernel = int(rng.choice([1, 3, 5, 7, 9]))
+    Wl = int(rng.integers(0, W + 1)) if rng.random() < 0.5 else 0
+    pool_mode = int(rng.random() < 0.3)
+    lens = None
+    if rng.random() < 0.5:
+        lens = tuple(int(x) for x in rng.integers(B + 1, L + 1, size=Bt))
+    return NL, Bt, Hkv * G, Hkv, D, L, W, Wl, kernel, B, pool_mode, lens
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_shapes_and_options_match_oracle(laq, seed):
+    NL, Bt, Hq, Hkv, D, L, W, Wl, kernel, B, pool_mode, lens = _random_case(seed)
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=seed, kscale=1.0 + (seed % 3))
+    err, _ = compare_all_units(laq, q, k, v, W, kernel, B, local_window=Wl, pool_mode=pool_mode,
+                               seq_lens=lens)
+    assert err < SCORE_RTOL
+
+
 def test_variant_argument_checks(laq):
     q, k, v = rand_inputs(1, 1, 4, 2, 128, 300, 8, seed=4)
     for kw in ({"pool_mode": 2}, {"pool_mode": -1}, {"score_mode": 2}):
