@@ -92,9 +92,9 @@ static laq_status check_strides_vo(const laq_params* p, bool need_v) {
 
 int choose_tiles_per_task(const Dims& d) {
   const int n_tiles = (d.L + TILE_KEYS - 1) / TILE_KEYS;
-  // default: at most 16 tasks per unit and sweep, and at least 8 tiles per task
-  int t = d.tiles_per_task > 0 ? d.tiles_per_task : (n_tiles + 15) / 16;
-  if (d.tiles_per_task <= 0 && t < 8) t = 8;  // measured best on B200 with the default lag
+  // default, measured on B200: 16 tiles (2048 keys) per task; 8 for short prompts, so that a unit
+  // still splits into several tasks
+  int t = d.tiles_per_task > 0 ? d.tiles_per_task : (n_tiles >= 64 ? 16 : 8);
   if (t > n_tiles) t = n_tiles;
   return t;
 }

@@ -73,7 +73,6 @@ struct TcArgs {
   int n_slots;     // K stages = accumulator buffers (4, or 2 when a buffer takes 256 columns)
   int slot_shift;  // log2(n_slots)
   int tb_cols;     // TMEM columns per accumulator buffer (128 or 256)
-  int dup;         // 1 when M <= 64: sweep 1 holds every query row twice, on lanes r and 64 + r
   SeqLens sl;      // per-prompt lengths (n = 0: every prompt holds L positions)
 };
 
@@ -399,6 +398,8 @@ __device__ __forceinline__ void stats_cols64(uint32_t taddr, float c, float& m, 
 }
 
 // ------------------------------------------------------------------ the kernel
+// kDup: M <= 64, sweep 1 holds every query row twice (on TMEM lanes r and 64 + r).
+template <bool kDup>
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
                 const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ TcArgs a) {
@@ -508,12 +509,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
           const uint32_t qs = qcount & 1u;
           if (!mbar_wait(a, ctl, smem_u32(&ctl->q_empty[qs]), ((qcount >> 1) & 1u) ^ 1u, 3)) break;
           const uint32_t bar = smem_u32(&ctl->q_full[qs]);
-          mbar_expect_tx(bar, (uint32_t)a.M * 256u * (a.dup ? 2u : 1u));
+          mbar_expect_tx(bar, (uint32_t)a.M * 256u * (kDup ? 2u : 1u));
           const uint32_t dst = q_base + qs * q_stage_bytes;
           tma_load_5d(dst, &tmap_q, bar, 0, 0, task.h * a.G, task.b, task.layer);
           tma_load_5d(dst + (uint32_t)a.q_rows * 128u, &tmap_q, bar, 64, 0, task.h * a.G, task.b,
                       task.layer);
-          if (a.dup) {
+          if (kDup) {
             // a second copy of the rows, 64 rows (8192 bytes: the swizzle pattern repeats) further
             tma_load_5d(dst + 8192u, &tmap_q, bar, 0, 0, task.h * a.G, task.b, task.layer);
             tma_load_5d(dst + (uint32_t)a.q_rows * 128u + 8192u, &tmap_q, bar, 64, 0, task.h * a.G,
@@ -638,7 +639,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         float m = -1e30f, l = 0.f;
 #pragma unroll
         for (int g = 0; g < kSoftmaxWgs; ++g) merge_stat(m, l, ctl->stat[s][g][row]);
-        if (a.dup) {  // the second copy of the row saw the other key columns
+        if (kDup) {  // the second copy of the row saw the other key columns
 #pragma unroll
           for (int g = 0; g < kSoftmaxWgs; ++g) merge_stat(m, l, ctl->stat[s][g][64 + row]);
         }
@@ -731,7 +732,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
     // Sweep 1 with M <= 64: lanes 64.. hold a second copy of the rows, so the warps on lanes r and
     // 64 + r share row r's 64 key columns of this warpgroup (32 each) and all four quadrants of
     // the SM work; otherwise this thread's rows are row_in_wg and 128 + row_in_wg.
-    const int row_s1 = a.dup ? (quad & 1) * 32 + lane : row_in_wg;
+    const int row_s1 = kDup ? (quad & 1) * 32 + lane : row_in_wg;
     const uint32_t col_d = 64u * (uint32_t)half + 32u * (uint32_t)(quad >> 1);  // dup: my 32 columns
     const int qi0 = row_s1 % a.W, qi1 = (128 + row_in_wg) % a.W;  // query index inside its head
     // Tiles are numbered through all tasks of this CTA; pair p owns tiles p, p + 2, ... A parity
@@ -776,9 +777,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         if (task.sweep == 0) {
           const int valid = min(TILE_KEYS, Lu - key0);
           // row blocks beyond the unit's rows are skipped (warp-uniform)
-          const bool rows0 = (a.dup ? (quad & 1) : quad) * 32 < a.M;
+          const bool rows0 = (kDup ? (quad & 1) : quad) * 32 < a.M;
           const bool rows1 = RB == 2 && 128 + quad * 32 < a.M;
-          if (a.dup) {
+          if (kDup) {
             if (!rows0) {
               release_buffer(empty_bar, lane);
             } else if (valid == TILE_KEYS && key0 + TILE_KEYS <= Lu - a.W_local) {
@@ -968,7 +969,7 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   a.n_slots = wide ? 2 : 4;
   a.slot_shift = wide ? 1 : 2;
   a.tb_cols = wide ? 256 : 128;
-  a.dup = w.M_pad <= 64 ? 1 : 0;
+  const bool dup = w.M_pad <= 64;  // sweep 1 holds every query row twice, on lanes r and 64 + r
 
   CUtensorMap tmap_q, tmap_k;
   const uint64_t qdims[5] = {128, (uint64_t)d.W, (uint64_t)d.Hq, (uint64_t)d.Bt, (uint64_t)d.NL};
@@ -981,14 +982,15 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
     return score_simt_launch(p, d, w, q, k, ws, stream, launches);  // layout TMA cannot describe
 
   const size_t smem = kCtlBytes + 2u * (size_t)a.q_rows * 256u + (size_t)a.n_slots * kKStageBytes;
-  if (cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)smem) != cudaSuccess)
+  auto kernel = dup ? score_tc_kernel<true> : score_tc_kernel<false>;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+      cudaSuccess)
     return LAQ_ERR_CUDA;
   // the softmax warpgroups add their shares into the column sums, which therefore start at zero
   if (cudaMemsetAsync(a.colsum, 0, (size_t)d.U * w.L_pad * sizeof(float), stream) != cudaSuccess)
     return LAQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.total_tickets < (uint32_t)sms ? a.total_tickets : (uint32_t)sms);
-  score_tc_kernel<<<grid, kThreads, smem, stream>>>(tmap_q, tmap_k, a);
+  kernel<<<grid, kThreads, smem, stream>>>(tmap_q, tmap_k, a);
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;
 }
