@@ -69,10 +69,6 @@ struct TcArgs {
   int32_t* cnt;
   float2* part;
   float* colsum;
-  int q_rows;      // rows allocated per 64-column half of a Q stage (128 or 256)
-  int n_slots;     // K stages = accumulator buffers (4, or 2 when a buffer takes 256 columns)
-  int slot_shift;  // log2(n_slots)
-  int tb_cols;     // TMEM columns per accumulator buffer (128 or 256)
   SeqLens sl;      // per-prompt lengths (n = 0: every prompt holds L positions)
 };
 
@@ -399,18 +395,24 @@ __device__ __forceinline__ void stats_cols64(uint32_t taddr, float c, float& m, 
 
 // ------------------------------------------------------------------ the kernel
 // kDup: M <= 64, sweep 1 holds every query row twice (on TMEM lanes r and 64 + r).
-template <bool kDup>
+// kWide: 128 < M <= 256, two row blocks per tile, so an accumulator buffer takes 256 TMEM columns
+// and there are two K stages / buffers instead of four.
+template <bool kDup, bool kWide>
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
                 const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ TcArgs a) {
+  constexpr uint32_t kQRows = kWide ? 256u : 128u;   // rows per 64-dim half of a Q stage
+  constexpr uint32_t kSlotShift = kWide ? 1u : 2u;   // log2 of the K stages = accumulator buffers
+  constexpr uint32_t kTbCols = kWide ? 256u : 128u;  // TMEM columns per accumulator buffer
+  constexpr int RB = kWide ? 2 : 1;                  // 128-row blocks per tile in sweep 1
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   Ctl* ctl = reinterpret_cast<Ctl*>(smem_raw);
   const uint32_t smem_base = smem_u32(smem_raw);
-  const uint32_t q_stage_bytes = (uint32_t)a.q_rows * 256u;
+  const uint32_t q_stage_bytes = kQRows * 256u;
   const uint32_t q_base = smem_base + kCtlBytes;
   const uint32_t k_base = q_base + 2u * q_stage_bytes;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t slot_mask = (uint32_t)a.n_slots - 1u;
+  constexpr uint32_t slot_mask = (1u << kSlotShift) - 1u;
 
   if ((smem_base & 1023u) != 0) {  // the swizzled stages need a 1024-byte aligned base
     if (threadIdx.x == 0 && atomicCAS(&a.hdr[HDR_STATUS], 0, (int)LAQ_ERR_INTERNAL) == 0)
@@ -512,12 +514,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
           mbar_expect_tx(bar, (uint32_t)a.M * 256u * (kDup ? 2u : 1u));
           const uint32_t dst = q_base + qs * q_stage_bytes;
           tma_load_5d(dst, &tmap_q, bar, 0, 0, task.h * a.G, task.b, task.layer);
-          tma_load_5d(dst + (uint32_t)a.q_rows * 128u, &tmap_q, bar, 64, 0, task.h * a.G, task.b,
+          tma_load_5d(dst + kQRows * 128u, &tmap_q, bar, 64, 0, task.h * a.G, task.b,
                       task.layer);
           if (kDup) {
             // a second copy of the rows, 64 rows (8192 bytes: the swizzle pattern repeats) further
             tma_load_5d(dst + 8192u, &tmap_q, bar, 0, 0, task.h * a.G, task.b, task.layer);
-            tma_load_5d(dst + (uint32_t)a.q_rows * 128u + 8192u, &tmap_q, bar, 64, 0, task.h * a.G,
+            tma_load_5d(dst + kQRows * 128u + 8192u, &tmap_q, bar, 64, 0, task.h * a.G,
                         task.b, task.layer);
           }
           ++qcount;
@@ -529,7 +531,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         for (int i = 0; i < task.n_tiles; ++i) {
           const uint32_t s = kcount & slot_mask;
           // the stage is free once the MMAs of the tile that used it last have completed
-          if (!mbar_wait(a, ctl, smem_u32(&ctl->mma_done[s]), ((kcount >> a.slot_shift) & 1u) ^ 1u, 4)) {
+          if (!mbar_wait(a, ctl, smem_u32(&ctl->mma_done[s]), ((kcount >> kSlotShift) & 1u) ^ 1u, 4)) {
             ok = false;
             break;
           }
@@ -575,8 +577,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       uint32_t tc_base = 0, my_next = issuer, qc = 0, tk = 0;
       const uint32_t idesc_s1 = instr_desc(128, TILE_KEYS);
       const uint32_t idesc_s2 = instr_desc(128, a.M_pad);
-      const int RB = (a.M + 127) / 128;
-      const uint32_t q_half16 = (uint32_t)a.q_rows * 8u;  // (q_rows * 128 bytes) >> 4
+      const uint32_t q_half16 = kQRows * 8u;  // (q_rows * 128 bytes) >> 4
       const uint32_t k_lo0 = smem_desc_lo(k_base), q_lo0 = smem_desc_lo(q_base);
       bool ok = true;
       while (ok) {
@@ -590,7 +591,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         for (; i < task.n_tiles; i += 2) {
           const uint32_t tc = tc_base + (uint32_t)i;
           const uint32_t s = tc & slot_mask;
-          const uint32_t ph = (tc >> a.slot_shift) & 1u;
+          const uint32_t ph = (tc >> kSlotShift) & 1u;
           if (!mbar_wait(a, ctl, smem_u32(&ctl->k_full[s]), ph, 12) ||
               !mbar_wait(a, ctl, smem_u32(&ctl->tmem_empty[s]), ph ^ 1u, 13)) {
             ok = false;
@@ -598,7 +599,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
           }
           tc_fence_after();
           const uint32_t k_lo = k_lo0 + s * (kKStageBytes >> 4);
-          const uint32_t d_tmem = tmem_base + s * (uint32_t)a.tb_cols;
+          const uint32_t d_tmem = tmem_base + s * kTbCols;
           // k-step kk covers dims [16 kk, 16 kk + 16): 32 bytes inside the 64-dim half (kk >> 2)
           if (task.sweep == 0) {
             for (int rb = 0; rb < RB; ++rb) {
@@ -723,7 +724,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
     const int row_in_wg = quad * 32 + lane;  // TMEM lane this thread reads
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const float c = a.scale_log2;
-    const int RB = (a.M + 127) / 128;
     // sweep 2: this warpgroup's share of the M_pad / 32 row chunks
     const int n_chunks2 = a.M_pad / 32;
     const int ch_lo = half == 0 ? 0 : (n_chunks2 + 1) / 2;
@@ -764,21 +764,21 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       for (; i < task.n_tiles; i += 2) {
         const uint32_t tc = tc_base + (uint32_t)i;
         const uint32_t s = tc & slot_mask;
-        if (!mbar_wait(a, ctl, smem_u32(&ctl->mma_done[s]), (tc >> a.slot_shift) & 1u, 21)) {
+        if (!mbar_wait(a, ctl, smem_u32(&ctl->mma_done[s]), (tc >> kSlotShift) & 1u, 21)) {
           ok = false;
           break;
         }
         __syncwarp();
         tc_fence_after();
         const int key0 = (task.tile0 + i) * TILE_KEYS;
-        const uint32_t taddr = lane_addr + s * (uint32_t)a.tb_cols;
+        const uint32_t taddr = lane_addr + s * kTbCols;
         const uint32_t empty_bar = smem_u32(&ctl->tmem_empty[s]);
         float v[32];
         if (task.sweep == 0) {
           const int valid = min(TILE_KEYS, Lu - key0);
           // row blocks beyond the unit's rows are skipped (warp-uniform)
           const bool rows0 = (kDup ? (quad & 1) : quad) * 32 < a.M;
-          const bool rows1 = RB == 2 && 128 + quad * 32 < a.M;
+          const bool rows1 = kWide && 128 + quad * 32 < a.M;
           if (kDup) {
             if (!rows0) {
               release_buffer(empty_bar, lane);
@@ -965,10 +965,7 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   a.colsum = (float*)(ws + w.off_colsum);
   a.sl = d.sl;
   const bool wide = d.M > 128;
-  a.q_rows = wide ? 256 : 128;
-  a.n_slots = wide ? 2 : 4;
-  a.slot_shift = wide ? 1 : 2;
-  a.tb_cols = wide ? 256 : 128;
+  const int q_rows = wide ? 256 : 128, n_slots = wide ? 2 : 4;
   const bool dup = w.M_pad <= 64;  // sweep 1 holds every query row twice, on lanes r and 64 + r
 
   CUtensorMap tmap_q, tmap_k;
@@ -981,8 +978,9 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   if (!make_map(&tmap_q, q, qdims, qstr, qbox) || !make_map(&tmap_k, k, kdims, kstr, kbox))
     return score_simt_launch(p, d, w, q, k, ws, stream, launches);  // layout TMA cannot describe
 
-  const size_t smem = kCtlBytes + 2u * (size_t)a.q_rows * 256u + (size_t)a.n_slots * kKStageBytes;
-  auto kernel = dup ? score_tc_kernel<true> : score_tc_kernel<false>;
+  const size_t smem = kCtlBytes + 2u * (size_t)q_rows * 256u + (size_t)n_slots * kKStageBytes;
+  auto kernel = dup ? score_tc_kernel<true, false>
+                    : (wide ? score_tc_kernel<false, true> : score_tc_kernel<false, false>);
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
       cudaSuccess)
     return LAQ_ERR_CUDA;
