@@ -633,6 +633,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       if (!next_task(a, ctl, tk, lane, false, 30, task)) break;
       if (task.sweep < 0) break;
       if (task.sweep != 0) continue;
+      // The column sums of this task's keys start at zero: sweep 2 adds into them with two
+      // red.global per key. Zeroed here, before the fence and the counter bump below, they are
+      // visible to every sweep-2 task of the unit, which waits for that counter.
+      {
+        float4* cz = reinterpret_cast<float4*>(a.colsum + (int64_t)task.unit * a.L_pad +
+                                               (int64_t)task.tile0 * TILE_KEYS);
+        const int n4 = task.n_tiles * (TILE_KEYS / 4);
+        for (int i = lane; i < n4; i += 32) cz[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
       const uint32_t s = sc % kStatSlots;
       if (!mbar_wait(a, ctl, smem_u32(&ctl->stat_full[s]), (sc / kStatSlots) & 1u, 31)) break;
       float2* dst = a.part + ((int64_t)task.unit * a.n_part + task.chunk) * a.M_pad;
@@ -983,9 +992,6 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
                     : (wide ? score_tc_kernel<false, true> : score_tc_kernel<false, false>);
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
       cudaSuccess)
-    return LAQ_ERR_CUDA;
-  // the softmax warpgroups add their shares into the column sums, which therefore start at zero
-  if (cudaMemsetAsync(a.colsum, 0, (size_t)d.U * w.L_pad * sizeof(float), stream) != cudaSuccess)
     return LAQ_ERR_CUDA;
   const unsigned grid = (unsigned)(a.total_tickets < (uint32_t)sms ? a.total_tickets : (uint32_t)sms);
   kernel<<<grid, kThreads, smem, stream>>>(tmap_q, tmap_k, a);
