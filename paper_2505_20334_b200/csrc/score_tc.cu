@@ -37,6 +37,10 @@
                               // measured 4 % slower with 4 tiles, the four-stage ring already covers the latency)
 #endif
 
+#ifndef LAQ_WAIT_HINT_NS
+#define LAQ_WAIT_HINT_NS 2000  // longest hardware suspension of one mbarrier poll
+#endif
+
 namespace laq {
 namespace {
 
@@ -131,6 +135,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       "selp.u32 %0, 1, 0, p;\n}"
       : "=r"(ok)
       : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// The same, letting the hardware suspend the thread for up to `ns` nanoseconds while the phase is
+// incomplete (it resumes as soon as the phase completes), so that a long wait polls rarely.
+__device__ __forceinline__ bool mbar_try_wait_for(uint32_t bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(ns)
       : "memory");
   return ok != 0;
 }
@@ -250,7 +267,7 @@ __device__ __forceinline__ bool mbar_wait(const TcArgs& a, Ctl* ctl, uint32_t ba
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t spins = 0;
-  while (!mbar_try_wait(bar, parity)) {
+  while (!mbar_try_wait_for(bar, parity, LAQ_WAIT_HINT_NS)) {
     if ((++spins & 63u) == 0) {
       if (ctl->abort) return false;
       if (clock64() - t0 > kTimeoutCycles) {
