@@ -69,7 +69,7 @@ extern "C" {
 typedef enum {
   LAQ_OK = 0,
   LAQ_ERR_INVALID_ARG = 1, /* null pointer, bad size relation, misaligned pointer or stride */
-  LAQ_ERR_UNSUPPORTED = 2, /* a valid problem this build has no kernel for (e.g. head_dim != 128) */
+  LAQ_ERR_UNSUPPORTED = 2, /* a valid problem this build has no kernel for (e.g. more than 256 rows) */
   LAQ_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or smaller than laq_workspace_bytes() */
   LAQ_ERR_CUDA = 4,        /* a CUDA runtime or driver call failed */
   LAQ_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out (see laq_last_device_status) */
@@ -93,7 +93,7 @@ typedef struct {
   int32_t batch;       /* Bt >= 1 */
   int32_t n_q_heads;   /* Hq, a multiple of n_kv_heads */
   int32_t n_kv_heads;  /* Hkv >= 1; query head h reads KV head h / G */
-  int32_t head_dim;    /* D; 128 is the supported value */
+  int32_t head_dim;    /* D, a multiple of 8 up to 256; 128 takes the tensor-core path */
   int32_t prompt_len;  /* L */
   int32_t window_len;  /* W >= 1 lookahead queries per query head; G*W <= 256 */
   int32_t keep_tail;   /* R, 0 <= R < B: last R positions always kept and never scored */
@@ -102,7 +102,8 @@ typedef struct {
   int32_t budget;      /* B, R < B < L */
   float softmax_scale; /* 0 selects 1/sqrt(head_dim) */
   /* Scheduling knobs of the scoring kernel; 0 lets the library choose. */
-  int32_t tiles_per_task;  /* 128-key tiles per scoring task (a task = one sweep over a key chunk) */
+  int32_t tiles_per_task;  /* 128-key tiles per scoring task (a task = one sweep over a key chunk);
+                            * it also sets the workspace size, so set it before laq_workspace_bytes */
   int32_t sched_lag_tasks; /* how many tasks the column-sum sweep trails the statistics sweep */
   /* LAQ++ (Eq. 5, unified window W u Q): the first local_window of each head's window_len queries
    * are the queries of the last local_window prompt positions (query i at position
