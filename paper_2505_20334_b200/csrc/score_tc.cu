@@ -91,6 +91,10 @@ struct Ctl {
   uint64_t k_full[kMaxSlots];
   // Tile t uses K stage t mod n_slots and accumulator buffer t mod n_slots, so one barrier per
   // slot tells the producer that the stage is free and the softmax warps that the logits are ready.
+  // n_slots is even: tiles t and t - n_slots then belong to the same MMA issuer and the same
+  // softmax pair, which is what makes the parity waits sound (a waiter is never two phases ahead).
+  // With five slots the second issuer can complete tile t - 2 before the first has issued tile
+  // t - 5, and the pair waiting for tile t then sees a stale phase (seen as a wait that ran out).
   uint64_t mma_done[kMaxSlots];
   uint64_t tmem_empty[kMaxSlots];
   uint64_t task_full[kTaskSlots], task_empty[kTaskSlots];
