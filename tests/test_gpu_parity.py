@@ -317,6 +317,19 @@ def test_prompts_of_different_lengths_match_oracle(laq, shape):
         assert (raw["idx"][:, b, :, B - W:].cpu().numpy() == np.arange(Lb - W, Lb)).all()
 
 
+def test_largest_ragged_batch_and_many_short_units(laq):
+    # 512 prompts (the most the per-prompt lengths take) of one or two tiles each, and the same
+    # geometry with equal lengths: many units with a single task each
+    NL, Bt, Hq, Hkv, D, L, W, kernel, B = 1, 512, 2, 1, 128, 200, 4, 3, 24
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=77)
+    rng = np.random.default_rng(77)
+    lens = tuple(int(x) for x in rng.integers(B + 1, L + 1, size=Bt))
+    err, _ = compare_all_units(laq, q, k, v, W, kernel, B, seq_lens=lens)
+    assert err < SCORE_RTOL
+    err, _ = compare_all_units(laq, q, k, v, W, kernel, B)
+    assert err < SCORE_RTOL
+
+
 def test_seq_lens_argument_checks(laq):
     q, k, v = rand_inputs(1, 2, 4, 2, 128, 300, 8, seed=5)
     for bad in ((300, 40), (301, 100), (300,)):     # not longer than the budget / too long / too few
