@@ -224,11 +224,22 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_reg_kernel(
     int kpool, float inv_k, int pool_max, const __grid_constant__ SelGeom g) {
   __shared__ uint32_t s_cnt[2][kSelWarps];
   __shared__ uint32_t s_gt[kSelWarps], s_eq[kSelWarps];
+  extern __shared__ __align__(16) float s_c[];  // the unit's column sums, [0, Ls) rounded up to 4
   const int64_t u = blockIdx.x;
-  const float* c = colsum + u * (int64_t)L_pad;
   const int Ls = unit_scored(g, u), Kb = g.Kb, R = g.R;
   int32_t* out = idx + u * (int64_t)g.B;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // One coalesced pass brings the column sums on chip (rows are 512-byte aligned and padded to
+  // a multiple of 128 floats); the pooling taps then read shared memory instead of L1/L2.
+  {
+    const float4* src = reinterpret_cast<const float4*>(colsum + u * (int64_t)L_pad);
+    float4* dst = reinterpret_cast<float4*>(s_c);
+    const int n4 = (Ls + 3) >> 2;
+#pragma unroll 8
+    for (int k = tid; k < n4; k += kSelThreads) dst[k] = __ldcs(src + k);
+  }
+  __syncthreads();
+  const float* c = s_c;
   const int base = warp * (kRegItems * 32) + lane;
   const int h = (kPoolStatic > 0 ? kPoolStatic : kpool) / 2;
 
@@ -356,9 +367,13 @@ laq_status pool_select_launch(const Dims& d, const float* colsum, int L_pad, flo
   if (d.Ls <= kRegItems * kSelThreads) {
     const float inv_k = 1.0f / (float)d.kpool;
     const unsigned grid = (unsigned)d.U;
-#define LAQ_LAUNCH_POOL_SELECT(KP)                                                         \
-  pool_select_reg_kernel<KP><<<grid, kSelThreads, 0, stream>>>(colsum, L_pad, pooled_out, idx, \
-                                                               d.kpool, inv_k, d.pool_max, g)
+    const size_t smem_c = (size_t)((d.Ls + 3) / 4 * 4) * sizeof(float);
+#define LAQ_LAUNCH_POOL_SELECT(KP)                                                                  \
+  if (cudaFuncSetAttribute(pool_select_reg_kernel<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                           (int)smem_c) != cudaSuccess)                                             \
+    return LAQ_ERR_CUDA;                                                                            \
+  pool_select_reg_kernel<KP><<<grid, kSelThreads, smem_c, stream>>>(colsum, L_pad, pooled_out, idx, \
+                                                                    d.kpool, inv_k, d.pool_max, g)
     switch (d.kpool) {
       case 1: LAQ_LAUNCH_POOL_SELECT(1); break;
       case 3: LAQ_LAUNCH_POOL_SELECT(3); break;
