@@ -330,6 +330,23 @@ def test_largest_ragged_batch_and_many_short_units(laq):
     assert err < SCORE_RTOL
 
 
+def test_host_buffer_entry_point_equals_device_run(laq):
+    # laq_evict_host: host tensors in, compressed cache out; same kernels, so the same bits
+    NL, Bt, Hq, Hkv, D, L, W, kernel, B = 2, 2, 8, 2, 128, 1100, 16, 7, 90
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=88)
+    for lens, Wl in ((None, 0), ((1100, 300), 8)):
+        dev = laq.evict(q.cuda(), k.cuda(), v.cuda(), B, pool_kernel=kernel, local_window=Wl, seq_lens=lens)
+        he = laq.HostEvictor(tuple(q.shape), tuple(k.shape), B, kernel, W, "cuda")
+        he.params.local_window = Wl
+        he.params.set_seq_lens(lens)
+        hk, hv, hidx = he.run(q.pin_memory(), k.pin_memory(), v.pin_memory())
+        torch.cuda.synchronize()
+        assert laq.laq_last_device_status(he.params, he.ws) == laq.LAQ_OK
+        assert torch.equal(hidx, dev["idx"].cpu())
+        assert torch.equal(hk.view(torch.int16), dev["k_out"].cpu().view(torch.int16))
+        assert torch.equal(hv.view(torch.int16), dev["v_out"].cpu().view(torch.int16))
+
+
 def test_seq_lens_argument_checks(laq):
     q, k, v = rand_inputs(1, 2, 4, 2, 128, 300, 8, seed=5)
     for bad in ((300, 40), (301, 100), (300,)):     # not longer than the budget / too long / too few
