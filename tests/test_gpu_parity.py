@@ -347,6 +347,41 @@ def test_host_buffer_entry_point_equals_device_run(laq):
         assert torch.equal(hv.view(torch.int16), dev["v_out"].cpu().view(torch.int16))
 
 
+def test_evict_can_be_captured_in_a_cuda_graph(laq):
+    # laq_evict only enqueues stream work (a memset and kernels): after one eager call it can be
+    # captured and replayed, and the replay gives the eager call's bits on new inputs
+    NL, Bt, Hq, Hkv, D, L, W, kernel, B = 2, 2, 8, 2, 128, 1500, 16, 7, 100
+    q, k, v = (t.cuda() for t in rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=91))
+    eager = laq.evict(q, k, v, B, pool_kernel=kernel, want_scores=True)
+    p, ws = eager["params"], eager["ws"]
+    k_out, v_out = torch.empty_like(eager["k_out"]), torch.empty_like(eager["v_out"])
+    idx, scores = torch.empty_like(eager["idx"]), torch.empty_like(eager["scores"])
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        laq.laq_evict(p, q, k, v, k_out, v_out, idx, scores, ws)   # warm-up on the capture stream
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            laq.laq_evict(p, q, k, v, k_out, v_out, idx, scores, ws)
+    torch.cuda.current_stream().wait_stream(side)
+    for t in (k_out, v_out, idx, scores):
+        t.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(idx, eager["idx"]) and torch.equal(scores, eager["scores"])
+    assert torch.equal(k_out.view(torch.int16), eager["k_out"].view(torch.int16))
+    # new contents in the same buffers: the replay follows them
+    q2, k2, v2 = (t.cuda() for t in rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=92))
+    q.copy_(q2); k.copy_(k2); v.copy_(v2)
+    graph.replay()
+    torch.cuda.synchronize()
+    again = laq.evict(q, k, v, B, pool_kernel=kernel, want_scores=True)
+    assert torch.equal(idx, again["idx"]) and torch.equal(scores, again["scores"])
+    assert torch.equal(v_out.view(torch.int16), again["v_out"].view(torch.int16))
+    assert laq.laq_last_device_status(p, ws) == laq.LAQ_OK
+
+
 def test_seq_lens_argument_checks(laq):
     q, k, v = rand_inputs(1, 2, 4, 2, 128, 300, 8, seed=5)
     for bad in ((300, 40), (301, 100), (300,)):     # not longer than the budget / too long / too few
