@@ -218,12 +218,15 @@ __device__ __forceinline__ void transpose32(uint32_t (&a)[32]) {
 }
 
 // kPoolStatic > 0 fixes the pooling kernel at compile time (unrolled taps); 0 takes it from `kpool`.
-template <int kPoolStatic>
-__global__ void __launch_bounds__(kSelThreads) pool_select_reg_kernel(
+// kThreads: block size (128 .. 1024); a unit of up to 32 * kThreads scored positions takes the
+// smallest one, so that several blocks of short units share an SM.
+template <int kPoolStatic, int kThreads>
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads) pool_select_reg_kernel(
     const float* __restrict__ colsum, int L_pad, float* pooled_out, int32_t* __restrict__ idx,
     int kpool, float inv_k, int pool_max, const __grid_constant__ SelGeom g) {
-  __shared__ uint32_t s_cnt[2][kSelWarps];
-  __shared__ uint32_t s_gt[kSelWarps], s_eq[kSelWarps];
+  constexpr int kWarps = kThreads / 32;
+  __shared__ uint32_t s_cnt[2][kWarps];
+  __shared__ uint32_t s_gt[kWarps], s_eq[kWarps];
   extern __shared__ __align__(16) float s_c[];  // the unit's column sums, [0, Ls) rounded up to 4
   const int64_t u = blockIdx.x;
   const int Ls = unit_scored(g, u), Kb = g.Kb, R = g.R;
@@ -236,7 +239,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_reg_kernel(
     float4* dst = reinterpret_cast<float4*>(s_c);
     const int n4 = (Ls + 3) >> 2;
 #pragma unroll 8
-    for (int k = tid; k < n4; k += kSelThreads) dst[k] = __ldcs(src + k);
+    for (int k = tid; k < n4; k += kThreads) dst[k] = __ldcs(src + k);
   }
   __syncthreads();
   const float* c = s_c;
@@ -287,7 +290,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_reg_kernel(
     uint32_t* slot = s_cnt[bit & 1];
     if (lane == 0) slot[warp] = n_warp;
     __syncthreads();
-    const uint32_t n = __reduce_add_sync(0xffffffffu, slot[lane]);
+    const uint32_t n = __reduce_add_sync(0xffffffffu, lane < kWarps ? slot[lane] : 0u);
     if (above + n >= (uint32_t)Kb) {
       theta |= 1u << bit;
       alive = ones;
@@ -326,7 +329,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_reg_kernel(
     gt_run += __popc(bg);
     eq_run += __popc(be);
   }
-  for (int t = tid; t < R; t += kSelThreads) out[Kb + t] = Ls + t;
+  for (int t = tid; t < R; t += kThreads) out[Kb + t] = Ls + t;
 }
 
 }  // namespace
@@ -368,12 +371,23 @@ laq_status pool_select_launch(const Dims& d, const float* colsum, int L_pad, flo
     const float inv_k = 1.0f / (float)d.kpool;
     const unsigned grid = (unsigned)d.U;
     const size_t smem_c = (size_t)((d.Ls + 3) / 4 * 4) * sizeof(float);
-#define LAQ_LAUNCH_POOL_SELECT(KP)                                                                  \
-  if (cudaFuncSetAttribute(pool_select_reg_kernel<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                           (int)smem_c) != cudaSuccess)                                             \
-    return LAQ_ERR_CUDA;                                                                            \
-  pool_select_reg_kernel<KP><<<grid, kSelThreads, smem_c, stream>>>(colsum, L_pad, pooled_out, idx, \
-                                                                    d.kpool, inv_k, d.pool_max, g)
+    // the smallest block whose 32 positions per thread cover the unit
+    const int threads = d.Ls <= 32 * 128 ? 128 : (d.Ls <= 32 * 256 ? 256 : (d.Ls <= 32 * 512 ? 512 : 1024));
+#define LAQ_LAUNCH_POOL_SELECT_T(KP, T)                                                               \
+  {                                                                                                   \
+    if (cudaFuncSetAttribute(pool_select_reg_kernel<KP, T>,                                           \
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_c) != cudaSuccess) \
+      return LAQ_ERR_CUDA;                                                                            \
+    pool_select_reg_kernel<KP, T><<<grid, T, smem_c, stream>>>(colsum, L_pad, pooled_out, idx, d.kpool, \
+                                                               inv_k, d.pool_max, g);                 \
+  }
+#define LAQ_LAUNCH_POOL_SELECT(KP)                     \
+  switch (threads) {                                   \
+    case 128: LAQ_LAUNCH_POOL_SELECT_T(KP, 128) break; \
+    case 256: LAQ_LAUNCH_POOL_SELECT_T(KP, 256) break; \
+    case 512: LAQ_LAUNCH_POOL_SELECT_T(KP, 512) break; \
+    default: LAQ_LAUNCH_POOL_SELECT_T(KP, 1024) break; \
+  }
     switch (d.kpool) {
       case 1: LAQ_LAUNCH_POOL_SELECT(1); break;
       case 3: LAQ_LAUNCH_POOL_SELECT(3); break;
@@ -382,6 +396,7 @@ laq_status pool_select_launch(const Dims& d, const float* colsum, int L_pad, flo
       default: LAQ_LAUNCH_POOL_SELECT(0); break;
     }
 #undef LAQ_LAUNCH_POOL_SELECT
+#undef LAQ_LAUNCH_POOL_SELECT_T
     *launches += 1;
     *done = true;
     return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;
