@@ -545,6 +545,11 @@ def sampled_parity(laq, cfg, budgets, units, device="cuda"):
             ws = laq.alloc_workspace(p, k.device)
         laq.laq_evict(p, q, k, v, k_out, v_out, idx, scores, ws)
         assert laq.laq_last_device_status(p, ws) == laq.LAQ_OK
+        # a second run hands the tasks to other SMs in another order; the bits must not change
+        scores2, idx2 = torch.empty_like(scores), torch.empty_like(idx)
+        laq.laq_evict(p, q, k, v, k_out, v_out, idx2, scores2, ws)
+        assert torch.equal(scores, scores2) and torch.equal(idx, idx2)
+        del scores2, idx2
         for u in units:
             h, b, n = u % Hkv, (u // Hkv) % Bt, u // (Hkv * Bt)
             qu, ku, vu = synth.unit_slices(cfg, inp, u)
