@@ -10,15 +10,20 @@
 // Both sweeps read the same K tile layout (TMA, 128-byte swizzle) and differ only in which operand
 // the tile is. Tickets alternate between the two sweeps, the second trailing the first by a fixed
 // number of tasks: far enough that a unit's statistics are final when its second sweep starts,
-// near enough that the second sweep re-reads K while it is still resident in L2. A sweep-2 task needs the unit's row statistics, i.e. the partial
-// statistics of every sweep-1 task of the unit; those tasks have smaller tickets, which running
-// CTAs already hold, so the order is deadlock-free for any grid size. Every wait is bounded.
+// near enough that the second sweep re-reads K while it is still resident in L2. A sweep-2 task
+// needs the unit's row statistics, i.e. the partial statistics of every sweep-1 task of the unit;
+// those tasks have smaller tickets, which running CTAs already hold, so the order is deadlock-free
+// for any grid size. Every wait is bounded.
+// For M <= 64 sweep 1 holds the query rows twice (TMEM lanes r and 64 + r) and the warps on the
+// two copies split the key columns; for 128 < M <= 256 a tile has two row blocks and takes a
+// 256-column accumulator buffer (two K stages / buffers instead of four).
 //
 // Warp roles (768 threads):
 //   warp 0       ticket fetch + TMA producer (one lane)
 //   warps 1, 20  tcgen05.mma issuers for alternate tiles (one lane each); warp 1 owns the TMEM
-//   warp 2       statistics out: merges the warpgroups' (shift, sum) of a finished sweep-1 task,
-//                writes the task's partial to global memory and bumps the unit's counter
+//   warp 2       statistics out: zeroes the column sums of a sweep-1 task's keys, merges the
+//                warpgroups' (shift, sum) of the finished task, writes the task's partial to
+//                global memory and bumps the unit's counter
 //   warps 3, 21-23  statistics in: for a sweep-2 task, wait for the unit's counter, merge the
 //                unit's partials into -b_r and hands them to the softmax warps in shared memory
 //   warps 4-19   four softmax warpgroups in two pairs. Pair p takes the tiles t with t mod 2 == p;
