@@ -408,15 +408,16 @@ __device__ __noinline__ float2 stats_cols_ragged(uint32_t taddr, int valid_max, 
 
 // Sweep 1, this warpgroup's 64 key columns of one row block of a full tile. If `release`, the
 // accumulator buffer is handed back to the MMA warp as soon as the last chunk is in registers.
+template <int kPoly>
 __device__ __forceinline__ void stats_cols64(uint32_t taddr, float c, float& m, float& l, float* v,
                                              bool release, uint32_t empty_bar, int lane) {
   tmem_ld32(taddr, v);
   tmem_ld_wait(v);
-  stats_chunk<LAQ_POLY_PAIRS_S1>(v, c, m, l);
+  stats_chunk<kPoly>(v, c, m, l);
   tmem_ld32(taddr + 32u, v);
   tmem_ld_wait(v);
   if (release) release_buffer(empty_bar, lane);
-  stats_chunk<LAQ_POLY_PAIRS_S1>(v, c, m, l);
+  stats_chunk<kPoly>(v, c, m, l);
 }
 
 // ------------------------------------------------------------------ the kernel
@@ -427,6 +428,8 @@ template <bool kDup, bool kWide>
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
                 const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ TcArgs a) {
+  // share of sweep 1's exponentials on the FMA pipe: measured to pay only for 64 < M <= 128
+  constexpr int kPolyS1 = (kDup || kWide) ? 0 : LAQ_POLY_PAIRS_S1;
   constexpr uint32_t kQRows = kWide ? 256u : 128u;   // rows per 64-dim half of a Q stage
   constexpr uint32_t kSlotShift = kWide ? 1u : 2u;   // log2 of the K stages = accumulator buffers
   constexpr uint32_t kTbCols = kWide ? 256u : 128u;  // TMEM columns per accumulator buffer
@@ -821,7 +824,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
               tmem_ld32(taddr + col_d, v);
               tmem_ld_wait(v);
               release_buffer(empty_bar, lane);
-              stats_chunk<LAQ_POLY_PAIRS_S1>(v, c, m0, l0);
+              stats_chunk<kPolyS1>(v, c, m0, l0);
             } else {
               const int vq = min(32, valid - (int)col_d);
               const float2 r =
@@ -832,8 +835,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
             }
           } else if (valid == TILE_KEYS && key0 + TILE_KEYS <= Lu - a.W_local) {
             // every column is a real key that every row sees
-            if (rows0) stats_cols64(taddr + col0, c, m0, l0, v, !rows1, empty_bar, lane);
-            if (rows1) stats_cols64(taddr + 128u + col0, c, m1, l1, v, true, empty_bar, lane);
+            if (rows0) stats_cols64<kPolyS1>(taddr + col0, c, m0, l0, v, !rows1, empty_bar, lane);
+            if (rows1) stats_cols64<kPolyS1>(taddr + 128u + col0, c, m1, l1, v, true, empty_bar, lane);
             if (!rows0) release_buffer(empty_bar, lane);
           } else {
             const int vh = min(64, valid - (int)col0);

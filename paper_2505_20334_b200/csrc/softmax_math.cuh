@@ -9,10 +9,12 @@
 
 #ifndef LAQ_POLY_PAIRS_S1
 // Of every 8 element pairs, how many take the FMA-pipe exp2 instead of the MUFU. Alone, the
-// arithmetic is fastest at 2-3 of 8 (MUFU-bound below, FMA-bound above); inside the kernel on a
-// B200 at its power cap the MUFU is the cheaper unit: 0 of 8 is 2 % faster than 2 of 8 and 6 %
-// faster than 4 of 8 (the GPU parity suite passes with 2 of 8 as well).
-#define LAQ_POLY_PAIRS_S1 0
+// arithmetic is fastest at 2-3 of 8 (MUFU-bound below, FMA-bound above). Inside the kernel on a
+// B200 (measured in alternating builds, 20- and 150-step runs): in sweep 1, 2 of 8 is 1.3 % faster
+// than 0 of 8 for 64 < M <= 128 (3 of 8 is equal to 0, 4 of 8 is slower), equal for M = 256 and
+// 1 % slower for M = 64, so the kernel uses it for 64 < M <= 128 only; in sweep 2, where every
+// chunk also loads its row offsets from shared memory, any share is slower.
+#define LAQ_POLY_PAIRS_S1 2
 #endif
 #ifndef LAQ_POLY_PAIRS_S2
 #define LAQ_POLY_PAIRS_S2 0  // same for sweep 2 (even)
