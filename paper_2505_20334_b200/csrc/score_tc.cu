@@ -979,18 +979,19 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   if (2 * n_stream >= 0x7fffffffll) return LAQ_ERR_UNSUPPORTED;
   a.total_tickets = (uint32_t)(2 * n_stream);
   // Sweep 2 trails sweep 1 by lag_tasks tasks. Too short and sweep-2 tasks wait for statistics
-  // that are not final yet; too long and K has left L2 when the second sweep reads it again.
-  // Measured on B200: the best distance is as much K as L2 still returns (about 52 MiB: 104-116
-  // tasks of 16 tiles at L = 32768, 208 tasks of 8 tiles at L = 16384), but never less than the
-  // tasks of one unit plus the tasks that half the SMs start while one task runs and its
-  // statistics travel (about 4 us); a 128-key tile takes 0.7-1.6 us per sweep depending on M.
+  // that are not final yet (a cliff: at L = 32768, 16-tile tasks, 100 tasks cost 10 %, 108 tasks
+  // 4 %); too long and K has left L2 when the second sweep reads it again (128 tasks = 64 MiB: 1 %).
+  // Measured best on B200: 120 tasks there, 208 tasks of 8 tiles at L = 16384. The rule: as much K
+  // as L2 still returns (about 52 MiB), but never less than the tasks of one unit plus the tasks
+  // that half the SMs start while one task runs and its statistics travel (about 5 us); a 128-key
+  // tile takes 0.7-1.6 us per sweep depending on M.
   int64_t lag_tasks = d.sched_lag_tasks;
   if (lag_tasks <= 0) {
     const int64_t task_bytes = (int64_t)a.tiles_per_task * TILE_KEYS * d.D * 2;
     const int64_t by_l2 = (52ll << 20) / task_bytes;
     const double tile_us = w.M_pad <= 64 ? 0.7 : (w.M_pad <= 128 ? 0.8 : 1.6);
     const int64_t by_latency =
-        a.tasks_per_unit + (int64_t)(0.5 * sms * (1.0 + 4.0 / (a.tiles_per_task * tile_us)) + 0.999);
+        a.tasks_per_unit + (int64_t)(0.5 * sms * (1.0 + 5.0 / (a.tiles_per_task * tile_us)) + 0.999);
     lag_tasks = by_l2 > by_latency ? by_l2 : by_latency;
   }
   if (lag_tasks < a.tasks_per_unit) lag_tasks = a.tasks_per_unit;
