@@ -32,7 +32,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one score_tc_kernel launch on this workload,
 # from the ncu capture summarised under profiles/ (None until one has been taken).
-NCU_TRAFFIC_BYTES = 9.88e9
+NCU_TRAFFIC_BYTES = 10.32e9
 NCU_TRAFFIC_BYTES_RAW = 8.68e9  # the same for score_raw_d128_kernel (--score-mode raw)
 
 
