@@ -56,11 +56,13 @@ constexpr int kSoftmaxWarps = 4 * kSoftmaxWgs;
 constexpr int kMmaWarpB = 4 + kSoftmaxWarps;  // index of the second MMA issuer's warp
 constexpr int kStatInWarps = 4;               // warp 3 and the warps after the second MMA issuer
 constexpr int kThreads = 32 * (kMmaWarpB + kStatInWarps);
-constexpr int kTaskSlots = 4;
+// ring depths of the task hand-off and of the two statistics hand-offs (measured: 6 and 3 are
+// 0.5-1 % faster than 4 and 2; deeper rings do not fit the shared memory next to the K stages)
+constexpr int kTaskSlots = 6;
 constexpr int kMaxSlots = 4;  // K stages in shared memory = TMEM accumulator buffers
-constexpr int kStatSlots = 2;
+constexpr int kStatSlots = 3;
 constexpr uint32_t kKStageBytes = TILE_KEYS * 128 * 2;  // 128 keys x 128 dims x bf16
-constexpr uint32_t kCtlBytes = 24576;
+constexpr uint32_t kCtlBytes = 34816;
 constexpr long long kTimeoutCycles = 4000000000LL;  // ~2 s: every device-side wait gives up after this
 constexpr float kLog2e = 1.4426950408889634f;
 // two MMA lanes, statistics-out warp, statistics-in warps, softmax warps
