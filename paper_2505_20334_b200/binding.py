@@ -346,4 +346,8 @@ class HostEvictor:
                 raise ValueError("laq_evict_host takes dense host tensors")
         laq_evict_host(self.params, q_host, k_host, v_host, self.h_k_out, self.h_v_out, self.h_idx,
                        self.staging, self.ws, stream)
+        # bytes that cross the bus towards the device: Q and K in full; V in full if it has to be
+        # staged, else only the kept rows, which the gather reads from the pinned host tensor
+        v_bytes = (self.h_v_out.numel() if v_host.is_pinned() else v_host.numel()) * 2
+        self.h2d_bytes = 2 * (q_host.numel() + k_host.numel()) + v_bytes
         return self.h_k_out, self.h_v_out, self.h_idx

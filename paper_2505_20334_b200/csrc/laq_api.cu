@@ -342,11 +342,27 @@ laq_status laq_evict_host(const laq_params* p, const void* q_host, const void* k
   laq_params_dense_strides(&dp);
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   char* sb = (char*)staging;
+  // Only the kept rows of V are ever read (step 6). If the host V is pinned memory that the GPU
+  // can address, the gather reads those rows straight from it and the full copy of V (half of the
+  // host-to-device traffic) is skipped; pageable memory is staged on the device like Q and K.
+  const void* v_dev = nullptr;
+  {
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, v_host) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
+        attr.devicePointer != nullptr && (reinterpret_cast<uintptr_t>(attr.devicePointer) & 15u) == 0)
+      v_dev = attr.devicePointer;
+    else
+      (void)cudaGetLastError();  // an unregistered pointer is not an error here
+  }
   if (cudaMemcpyAsync(sb + h.off_q, q_host, h.q_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
-      cudaMemcpyAsync(sb + h.off_k, k_host, h.kv_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
-      cudaMemcpyAsync(sb + h.off_v, v_host, h.kv_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+      cudaMemcpyAsync(sb + h.off_k, k_host, h.kv_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
     return LAQ_ERR_CUDA;
-  st = laq_evict(&dp, sb + h.off_q, sb + h.off_k, sb + h.off_v, sb + h.off_ko, sb + h.off_vo,
+  if (!v_dev) {
+    if (cudaMemcpyAsync(sb + h.off_v, v_host, h.kv_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+      return LAQ_ERR_CUDA;
+    v_dev = sb + h.off_v;
+  }
+  st = laq_evict(&dp, sb + h.off_q, sb + h.off_k, v_dev, sb + h.off_ko, sb + h.off_vo,
                  (int32_t*)(sb + h.off_idx), nullptr, ws, ws_bytes, cuda_stream);
   if (st != LAQ_OK) return st;
   if (cudaMemcpyAsync(k_out_host, sb + h.off_ko, h.out_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||

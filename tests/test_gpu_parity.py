@@ -339,12 +339,17 @@ def test_host_buffer_entry_point_equals_device_run(laq):
         he = laq.HostEvictor(tuple(q.shape), tuple(k.shape), B, kernel, W, "cuda")
         he.params.local_window = Wl
         he.params.set_seq_lens(lens)
-        hk, hv, hidx = he.run(q.pin_memory(), k.pin_memory(), v.pin_memory())
-        torch.cuda.synchronize()
-        assert laq.laq_last_device_status(he.params, he.ws) == laq.LAQ_OK
-        assert torch.equal(hidx, dev["idx"].cpu())
-        assert torch.equal(hk.view(torch.int16), dev["k_out"].cpu().view(torch.int16))
-        assert torch.equal(hv.view(torch.int16), dev["v_out"].cpu().view(torch.int16))
+        # pinned V: its kept rows are gathered straight from host memory; pageable V: staged
+        for v_host in (v.pin_memory(), v.clone()):
+            hk, hv, hidx = he.run(q.pin_memory(), k.pin_memory(), v_host)
+            torch.cuda.synchronize()
+            assert laq.laq_last_device_status(he.params, he.ws) == laq.LAQ_OK
+            assert torch.equal(hidx, dev["idx"].cpu())
+            assert torch.equal(hk.view(torch.int16), dev["k_out"].cpu().view(torch.int16))
+            assert torch.equal(hv.view(torch.int16), dev["v_out"].cpu().view(torch.int16))
+            assert he.h2d_bytes == 2 * (q.numel() + k.numel()) + 2 * (
+                hv.numel() if v_host.is_pinned() else v.numel())
+            hk.zero_(); hv.zero_(); hidx.zero_()
 
 
 def test_evict_can_be_captured_in_a_cuda_graph(laq):
