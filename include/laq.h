@@ -242,6 +242,8 @@ LAQ_API laq_status laq_recall(int64_t n_units, const int32_t* idx_pred, int32_t 
  * Only the kept rows of V are needed (step 6): when v_host is pinned (page-locked) memory that
  * the GPU can address, the gather reads those rows directly from it and V is not copied to the
  * device at all, which halves the host-to-device traffic; pageable v_host is staged like Q and K.
+ * Pinned k_out_host / v_out_host are likewise written by the gather directly instead of being
+ * staged and copied back.
  */
 LAQ_API size_t laq_host_staging_bytes(const laq_params* p);
 LAQ_API laq_status laq_evict_host(const laq_params* p, const void* q_host, const void* k_host,

@@ -317,6 +317,17 @@ static void plan_staging(const Dims& d, HostStaging* h) {
   h->total = off;
 }
 
+// Device address of a pinned (page-locked) host buffer that the GPU can access directly, 16-byte
+// aligned; NULL for pageable memory.
+static void* device_view_of_pinned(const void* host) {
+  cudaPointerAttributes attr;
+  if (cudaPointerGetAttributes(&attr, host) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
+      attr.devicePointer != nullptr && (reinterpret_cast<uintptr_t>(attr.devicePointer) & 15u) == 0)
+    return attr.devicePointer;
+  (void)cudaGetLastError();  // an unregistered pointer is not an error here
+  return nullptr;
+}
+
 size_t laq_host_staging_bytes(const laq_params* p) {
   Dims d;
   if (derive_dims(p, &d) != LAQ_OK) return 0;
@@ -345,15 +356,11 @@ laq_status laq_evict_host(const laq_params* p, const void* q_host, const void* k
   // Only the kept rows of V are ever read (step 6). If the host V is pinned memory that the GPU
   // can address, the gather reads those rows straight from it and the full copy of V (half of the
   // host-to-device traffic) is skipped; pageable memory is staged on the device like Q and K.
-  const void* v_dev = nullptr;
-  {
-    cudaPointerAttributes attr;
-    if (cudaPointerGetAttributes(&attr, v_host) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
-        attr.devicePointer != nullptr && (reinterpret_cast<uintptr_t>(attr.devicePointer) & 15u) == 0)
-      v_dev = attr.devicePointer;
-    else
-      (void)cudaGetLastError();  // an unregistered pointer is not an error here
-  }
+  // The same holds for the outputs: pinned K_out / V_out are written by the gather directly, in
+  // the same kernel that reads the V rows, so both directions of the bus work at once.
+  const void* v_dev = device_view_of_pinned(v_host);
+  void* ko_dev = device_view_of_pinned(k_out_host);
+  void* vo_dev = device_view_of_pinned(v_out_host);
   if (cudaMemcpyAsync(sb + h.off_q, q_host, h.q_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
       cudaMemcpyAsync(sb + h.off_k, k_host, h.kv_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
     return LAQ_ERR_CUDA;
@@ -362,11 +369,14 @@ laq_status laq_evict_host(const laq_params* p, const void* q_host, const void* k
       return LAQ_ERR_CUDA;
     v_dev = sb + h.off_v;
   }
-  st = laq_evict(&dp, sb + h.off_q, sb + h.off_k, v_dev, sb + h.off_ko, sb + h.off_vo,
-                 (int32_t*)(sb + h.off_idx), nullptr, ws, ws_bytes, cuda_stream);
+  st = laq_evict(&dp, sb + h.off_q, sb + h.off_k, v_dev, ko_dev ? ko_dev : sb + h.off_ko,
+                 vo_dev ? vo_dev : sb + h.off_vo, (int32_t*)(sb + h.off_idx), nullptr, ws, ws_bytes,
+                 cuda_stream);
   if (st != LAQ_OK) return st;
-  if (cudaMemcpyAsync(k_out_host, sb + h.off_ko, h.out_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
-      cudaMemcpyAsync(v_out_host, sb + h.off_vo, h.out_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+  if ((!ko_dev && cudaMemcpyAsync(k_out_host, sb + h.off_ko, h.out_bytes, cudaMemcpyDeviceToHost,
+                                  stream) != cudaSuccess) ||
+      (!vo_dev && cudaMemcpyAsync(v_out_host, sb + h.off_vo, h.out_bytes, cudaMemcpyDeviceToHost,
+                                  stream) != cudaSuccess) ||
       (idx_host && cudaMemcpyAsync(idx_host, sb + h.off_idx, h.idx_bytes, cudaMemcpyDeviceToHost,
                                    stream) != cudaSuccess))
     return LAQ_ERR_CUDA;

@@ -350,6 +350,16 @@ def test_host_buffer_entry_point_equals_device_run(laq):
             assert he.h2d_bytes == 2 * (q.numel() + k.numel()) + 2 * (
                 hv.numel() if v_host.is_pinned() else v.numel())
             hk.zero_(); hv.zero_(); hidx.zero_()
+        # pageable outputs are staged on the device and copied back
+        pk, pv, pidx = torch.zeros_like(hk, pin_memory=False), torch.zeros_like(hv, pin_memory=False), \
+            torch.zeros_like(hidx, pin_memory=False)
+        assert not pk.is_pinned()
+        laq.laq_evict_host(he.params, q.pin_memory(), k.pin_memory(), v.clone(), pk, pv, pidx,
+                           he.staging, he.ws)
+        torch.cuda.synchronize()
+        assert torch.equal(pidx, dev["idx"].cpu())
+        assert torch.equal(pk.view(torch.int16), dev["k_out"].cpu().view(torch.int16))
+        assert torch.equal(pv.view(torch.int16), dev["v_out"].cpu().view(torch.int16))
 
 
 def test_evict_can_be_captured_in_a_cuda_graph(laq):
