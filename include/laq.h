@@ -69,7 +69,7 @@ extern "C" {
 typedef enum {
   LAQ_OK = 0,
   LAQ_ERR_INVALID_ARG = 1, /* null pointer, bad size relation, misaligned pointer or stride */
-  LAQ_ERR_UNSUPPORTED = 2, /* a valid problem this build has no kernel for (e.g. more than 256 rows) */
+  LAQ_ERR_UNSUPPORTED = 2, /* a valid problem the library has no kernel for (e.g. more than 256 rows) */
   LAQ_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or smaller than laq_workspace_bytes() */
   LAQ_ERR_CUDA = 4,        /* a CUDA runtime or driver call failed */
   LAQ_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out (see laq_last_device_status) */

@@ -17,7 +17,7 @@
  * heads and queries, budget nestedness, planted key kept.
  * Parity unpinned by the paper: the softmax reading of Eq. 4, the sum over the GQA group, the
  * average pool with zero padding and divisor k, and the retained tail are conventions fixed by
- * the benchmark spec, not by a value the paper prints.
+ * the problem statement this oracle was written for, not by a value the paper prints.
  */
 #include <math.h>
 #include <stdint.h>
