@@ -34,21 +34,25 @@
  *               followed by the tail Ls..L-1
  *   6. gather   K_out[t] = K[idx[t]],  V_out[t] = V[idx[t]]
  *
- * Conventions common to every entry point
- *   - Every data pointer is a DEVICE pointer owned by the caller. Nothing is allocated, retained
- *     or freed by the library; scratch memory is the caller's workspace `ws` of at least
- *     laq_workspace_bytes() bytes, 256-byte aligned. A workspace may be reused by later calls on
- *     the same stream; two calls that overlap on the GPU need two workspaces.
+ * Conventions common to every entry point (the exceptions are named where they apply)
+ *   - Data pointers are DEVICE pointers owned by the caller, except in laq_evict_host, whose
+ *     tensors live in host memory. The library allocates, retains and frees no device memory;
+ *     scratch memory is the caller's workspace `ws` of at least laq_workspace_bytes() bytes,
+ *     256-byte aligned. A workspace may be reused by later calls on the same stream; two calls
+ *     that overlap on the GPU need two workspaces. The one exception is laq_score_static, whose
+ *     scratch is a fixed array inside the library image that all of its calls share.
  *   - Q, K, V, K_out, V_out hold bf16; the innermost (head_dim) stride is 1 and every other
  *     stride, given in ELEMENTS in laq_params, is a multiple of 8 (16 bytes). Base pointers are
  *     16-byte aligned.
  *   - Calls validate on the host, enqueue kernels on `cuda_stream` (a cudaStream_t passed as
  *     void*; NULL = the legacy default stream) and return without synchronising. A non-OK status
- *     means nothing was enqueued, except LAQ_ERR_CUDA from a failed launch.
+ *     means nothing was enqueued, except LAQ_ERR_CUDA from a failed launch or copy.
  *   - Device-side waits are bounded. If one runs out the kernel records it in the workspace and
  *     finishes; laq_last_device_status() reads that record back (it synchronises the stream).
- *   - No exceptions cross the boundary; the library keeps no global mutable state apart from
- *     cached per-device attributes.
+ *   - No exceptions cross the boundary. Mutable state kept inside the library: cached per-device
+ *     attributes; two per-host-thread instrumentation values (the stage events of
+ *     laq_set_stage_events and the counter behind laq_last_launch_count); the cached address and
+ *     the contents of laq_score_static's scratch array.
  */
 #ifndef LAQ_H_
 #define LAQ_H_
@@ -137,7 +141,8 @@ typedef struct {
 LAQ_API void laq_params_dense_strides(laq_params* p);
 
 /* Bytes of caller-provided device scratch that laq_score / laq_evict need for `p`
- * (0 if `p` is invalid). laq_select and laq_compact need none. */
+ * (0 if `p` is invalid). laq_select, laq_compact and laq_recall need none and take no workspace
+ * argument. */
 LAQ_API size_t laq_workspace_bytes(const laq_params* p);
 
 /*
@@ -160,16 +165,20 @@ LAQ_API laq_status laq_score(const laq_params* p, const void* q, const void* k, 
  * for hosts that give all device memory to their own pool at start-up and may not call the
  * driver's allocator afterwards -- an inference server whose allocator owns the GPU, a plugin
  * that receives tensors and a stream but no allocator, a latency-critical loop that cannot take
- * the device-wide synchronisation of an allocation. The call itself performs no allocation of
- * any kind.
+ * the device-wide synchronisation of an allocation. After one warm-up call per device the call
+ * allocates nothing: no cudaMalloc, no cudaFree, no allocating library routine. The warm-up call
+ * is different, because CUDA loads a library's kernels and device arrays lazily: the first call on
+ * a device is what makes the driver place the scratch array and the kernel code in that device's
+ * memory, so make it at start-up, before the host's own pool claims the GPU (on a GPU with no
+ * room left it fails with LAQ_ERR_CUDA), and outside any stream capture.
  *   q, k, scores   as for laq_score (device pointers; scores dense [NL][Bt][Hkv][L-R], fp32)
  * Limits and rules
  *   - The problem's scratch (per-unit counters, per-task row statistics and one fp32 column sum
  *     per key: roughly 4 bytes per cached key plus 8*M bytes per scoring task) must fit in
  *     LAQ_STATIC_SCRATCH_BYTES; otherwise LAQ_ERR_WORKSPACE is returned and nothing is enqueued.
  *     Larger problems can be scored in slices of layers with one call per slice.
- *   - The first call on a device looks up the array's device address (with that device current)
- *     and caches it; make that first call outside any stream capture.
+ *   - The first call on a device also looks up the array's device address (with that device
+ *     current) and caches it for later calls.
  *   - Every call uses the same array, which still holds the previous call's contents; the call
  *     clears the parts that must start at zero. Two calls that overlap on the GPU (different
  *     streams, or different host threads without ordering) race on it: order them.
@@ -266,6 +275,20 @@ LAQ_API laq_status laq_last_device_status(const laq_params* p, const void* ws, s
  * must outlive the calls that record them.
  */
 LAQ_API void laq_set_stage_events(void* score_begin, void* score_end);
+
+/*
+ * Instrumentation for benchmarks (no counterpart in the paper): synchronises `cuda_stream` and
+ * reads what the tensor-core scoring kernel of the last laq_score / laq_evict call on `ws`
+ * recorded about itself: the SM clock cycles and the wall-clock nanoseconds its first thread block
+ * ran for (the block is resident for the whole launch). cycles / nanoseconds is the SM clock the
+ * kernel really ran at; the board lowers it under load, so cycle counts and times are reported
+ * separately. Both read 0 if the call took another scoring path (head_dim other than 128, raw mode).
+ *   ws, ws_bytes   the workspace of that call (device)
+ *   sm_cycles, nanoseconds   HOST, out
+ * Errors: LAQ_ERR_INVALID_ARG, LAQ_ERR_CUDA.
+ */
+LAQ_API laq_status laq_last_kernel_clock(const void* ws, size_t ws_bytes, void* cuda_stream,
+                                         int64_t* sm_cycles, int64_t* nanoseconds);
 
 /* Kernel launches the most recent call on this host thread enqueued (for accounting). */
 LAQ_API int laq_last_launch_count(void);

@@ -29,7 +29,7 @@ EXPORTS = (
     "laq_params_dense_strides", "laq_workspace_bytes", "laq_score", "laq_select", "laq_compact",
     "laq_evict", "laq_last_device_status", "laq_last_launch_count", "laq_status_string",
     "laq_version", "laq_set_stage_events", "laq_host_staging_bytes", "laq_evict_host",
-    "laq_score_static", "laq_recall",
+    "laq_score_static", "laq_recall", "laq_last_kernel_clock",
 )
 
 
@@ -99,6 +99,9 @@ def _load() -> ctypes.CDLL:
     lib.laq_evict_host.restype = ctypes.c_int
     lib.laq_set_stage_events.argtypes = [vp, vp]
     lib.laq_set_stage_events.restype = None
+    lib.laq_last_kernel_clock.argtypes = [vp, sz, vp, ctypes.POINTER(ctypes.c_int64),
+                                          ctypes.POINTER(ctypes.c_int64)]
+    lib.laq_last_kernel_clock.restype = ctypes.c_int
     lib.laq_version.argtypes = []
     lib.laq_version.restype = ctypes.c_int
     return lib
@@ -231,6 +234,16 @@ def laq_evict(p: LaqParams, q, k, v, k_out, v_out, idx, scores, ws, stream=None,
 def laq_last_device_status(p: LaqParams, ws, stream=None) -> int:
     wp, wn = _ws_args(ws)
     return int(lib.laq_last_device_status(ctypes.byref(p), wp, wn, _stream(stream)))
+
+
+def laq_last_kernel_clock(ws, stream=None):
+    """(SM cycles, nanoseconds) the first block of the last tensor-core scoring launch on `ws` ran for."""
+    wp, wn = _ws_args(ws)
+    cyc, ns = ctypes.c_int64(0), ctypes.c_int64(0)
+    st = lib.laq_last_kernel_clock(wp, wn, _stream(stream), ctypes.byref(cyc), ctypes.byref(ns))
+    if st != LAQ_OK:
+        raise LaqError(st, "laq_last_kernel_clock")
+    return int(cyc.value), int(ns.value)
 
 
 def laq_last_launch_count() -> int:

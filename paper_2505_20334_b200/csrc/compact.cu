@@ -17,7 +17,7 @@ struct CompactArgs {
   int64_t vs_layer, vs_batch, vs_head, vs_pos;
   int64_t os_layer, os_batch, os_head, os_pos;
   int Bt, Hkv, B, dv, L;
-  int64_t total;  // U * B * dv
+  int64_t u0;  // first unit of this launch (units are launched in slabs of at most 65535)
 };
 
 // grid (row groups, units), block 256 threads = 16 half-warps. A half-warp copies one 256-byte
@@ -28,7 +28,7 @@ constexpr int kRowsInFlight = 4;
 constexpr int kRowsPerBlock = 16 * kRowsInFlight;
 
 __global__ void __launch_bounds__(256) compact_kernel(CompactArgs a) {
-  const int64_t u = blockIdx.y;
+  const int64_t u = a.u0 + blockIdx.y;
   const int h = (int)(u % a.Hkv);
   const int b = (int)((u / a.Hkv) % a.Bt);
   const int64_t layer = u / ((int64_t)a.Hkv * a.Bt);
@@ -85,12 +85,16 @@ laq_status compact_launch(const laq_params& p, const Dims& d, const void* k, con
   a.os_layer = p.o_stride_layer / 8; a.os_batch = p.o_stride_batch / 8;
   a.os_head = p.o_stride_head / 8;   a.os_pos = p.o_stride_pos / 8;
   a.Bt = d.Bt; a.Hkv = d.Hkv; a.B = d.B; a.dv = d.D / 8; a.L = d.L;
-  a.total = d.U * (int64_t)d.B * a.dv;
-  if (d.U > 65535) return LAQ_ERR_UNSUPPORTED;
-  compact_kernel<<<dim3((unsigned)((d.B + kRowsPerBlock - 1) / kRowsPerBlock), (unsigned)d.U), 256, 0,
-                   stream>>>(a);
-  *launches += 1;
-  return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;
+  // units sit on grid.y, which holds at most 65535 blocks
+  for (int64_t u0 = 0; u0 < d.U; u0 += 65535) {
+    a.u0 = u0;
+    const int64_t nu = d.U - u0 < 65535 ? d.U - u0 : 65535;
+    compact_kernel<<<dim3((unsigned)((d.B + kRowsPerBlock - 1) / kRowsPerBlock), (unsigned)nu), 256, 0,
+                     stream>>>(a);
+    *launches += 1;
+    if (cudaGetLastError() != cudaSuccess) return LAQ_ERR_CUDA;
+  }
+  return LAQ_OK;
 }
 
 }  // namespace laq

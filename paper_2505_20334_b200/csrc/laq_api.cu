@@ -67,7 +67,7 @@ laq_status derive_dims(const laq_params* p, Dims* d) {
   return derive_seq_lens(p, &d->sl);
 }
 
-static laq_status check_strides_qk(const laq_params* p) {
+laq_status check_strides_qk(const laq_params* p) {
   if (!mult8(p->q_stride_layer) || !mult8(p->q_stride_batch) || !mult8(p->q_stride_head) ||
       !mult8(p->q_stride_pos) || !mult8(p->k_stride_layer) || !mult8(p->k_stride_batch) ||
       !mult8(p->k_stride_head) || !mult8(p->k_stride_pos))
@@ -130,8 +130,10 @@ static bool use_tensor_core_path(const Dims& d) { return d.D == 128 && d.M <= 25
 static thread_local int g_last_launches = 0;
 static thread_local cudaEvent_t g_ev_begin = nullptr, g_ev_end = nullptr;
 
+void set_last_launch_count(int n) { g_last_launches = n; }
+
 // Steps 1-3 into the workspace's colsum array.
-static laq_status run_scoring(const laq_params* p, const Dims& d, const Workspace& w,
+laq_status run_scoring(const laq_params* p, const Dims& d, const Workspace& w,
                               const void* q, const void* k, char* ws, cudaStream_t stream,
                               int* launches) {
   // header and unit counters are contiguous: one clear
@@ -351,6 +353,12 @@ laq_status laq_evict_host(const laq_params* p, const void* q_host, const void* k
     return LAQ_ERR_WORKSPACE;
   laq_params dp = *p;
   laq_params_dense_strides(&dp);
+  // everything laq_evict would refuse is refused here, before the first copy is enqueued
+  {
+    Workspace w;
+    plan_workspace(d, choose_tiles_per_task(d), &w);
+    if ((st = check_ws(w, ws, ws_bytes)) != LAQ_OK) return st;
+  }
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   char* sb = (char*)staging;
   // Only the kept rows of V are ever read (step 6). If the host V is pinned memory that the GPU
@@ -394,6 +402,18 @@ laq_status laq_last_device_status(const laq_params* p, const void* ws, size_t ws
   if (cudaMemcpy(hdr, ws, sizeof hdr, cudaMemcpyDeviceToHost) != cudaSuccess) return LAQ_ERR_CUDA;
   if (hdr[HDR_STATUS] == 0) return LAQ_OK;
   return hdr[HDR_STATUS] == LAQ_ERR_TIMEOUT ? LAQ_ERR_TIMEOUT : LAQ_ERR_INTERNAL;
+}
+
+laq_status laq_last_kernel_clock(const void* ws, size_t ws_bytes, void* cuda_stream,
+                                 int64_t* sm_cycles, int64_t* nanoseconds) {
+  if (!ws || ws_bytes < HDR_WORDS * sizeof(int32_t) || !sm_cycles || !nanoseconds)
+    return LAQ_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return LAQ_ERR_CUDA;
+  int32_t hdr[HDR_WORDS];
+  if (cudaMemcpy(hdr, ws, sizeof hdr, cudaMemcpyDeviceToHost) != cudaSuccess) return LAQ_ERR_CUDA;
+  memcpy(sm_cycles, &hdr[HDR_CYCLES], sizeof(int64_t));
+  memcpy(nanoseconds, &hdr[HDR_NANOS], sizeof(int64_t));
+  return LAQ_OK;
 }
 
 void laq_set_stage_events(void* score_begin, void* score_end) {

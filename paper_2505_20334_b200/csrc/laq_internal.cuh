@@ -48,7 +48,10 @@ struct Workspace {
   int L_pad;   // L padded to a multiple of 128
 };
 
-enum { HDR_STATUS = 0, HDR_TICKET = 1, HDR_WHERE = 2, HDR_WORDS = 64 };
+// HDR_CYCLES / HDR_NANOS (two words each): SM clock cycles and wall-clock nanoseconds the first CTA
+// of the last tensor-core scoring launch ran for (instrumentation: their ratio is the SM clock the
+// kernel actually ran at, which the board's power management lowers under load).
+enum { HDR_STATUS = 0, HDR_TICKET = 1, HDR_WHERE = 2, HDR_CYCLES = 4, HDR_NANOS = 6, HDR_WORDS = 64 };
 
 // Keys per scoring task (a task = one sweep over KEYS_PER_TASK consecutive keys of one unit).
 constexpr int TILE_KEYS = 128;
@@ -56,6 +59,14 @@ constexpr int TILE_KEYS = 128;
 laq_status derive_dims(const laq_params* p, Dims* d);
 void plan_workspace(const Dims& d, int tiles_per_task, Workspace* w);
 int choose_tiles_per_task(const Dims& d);
+
+// Host-side checks and the scoring dispatch shared by every entry point that scores.
+laq_status check_strides_qk(const laq_params* p);
+// Steps 1-3 into the workspace's colsum array: clears the header and the unit counters, records
+// the caller's stage events around the scoring kernel and picks the back end.
+laq_status run_scoring(const laq_params* p, const Dims& d, const Workspace& w, const void* q,
+                       const void* k, char* ws, cudaStream_t stream, int* launches);
+void set_last_launch_count(int n);
 
 // Scoring back ends: both fill colsum (fp32 [U][L_pad]) on `stream`.
 // Tensor-core path (tcgen05 + TMA), head_dim 128, M <= 256.

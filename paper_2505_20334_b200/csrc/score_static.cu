@@ -38,8 +38,6 @@ laq_status static_scratch(void** out) {
   return LAQ_OK;
 }
 
-bool mult8(int64_t x) { return x > 0 && (x % 8) == 0; }
-
 }  // namespace
 }  // namespace laq
 
@@ -47,17 +45,14 @@ using namespace laq;
 
 extern "C" laq_status laq_score_static(const laq_params* p, const void* q, const void* k,
                                        float* scores, void* cuda_stream) {
+  set_last_launch_count(0);
   Dims d;
   laq_status st = derive_dims(p, &d);
   if (st != LAQ_OK) return st;
   if (!q || !k || !scores || (reinterpret_cast<uintptr_t>(q) & 15u) ||
       (reinterpret_cast<uintptr_t>(k) & 15u) || (reinterpret_cast<uintptr_t>(scores) & 3u))
     return LAQ_ERR_INVALID_ARG;
-  if (!mult8(p->q_stride_layer) || !mult8(p->q_stride_batch) || !mult8(p->q_stride_head) ||
-      !mult8(p->q_stride_pos) || !mult8(p->k_stride_layer) || !mult8(p->k_stride_batch) ||
-      !mult8(p->k_stride_head) || !mult8(p->k_stride_pos) || p->q_stride_pos < p->head_dim ||
-      p->k_stride_pos < p->head_dim)
-    return LAQ_ERR_INVALID_ARG;
+  if ((st = check_strides_qk(p)) != LAQ_OK) return st;
   Workspace w;
   plan_workspace(d, choose_tiles_per_task(d), &w);
   // everything up to and including the column sums is needed; the caller supplies the scores
@@ -66,13 +61,12 @@ extern "C" laq_status laq_score_static(const laq_params* p, const void* q, const
   if ((st = static_scratch(&base)) != LAQ_OK) return st;
   char* ws = static_cast<char*>(base);
   cudaStream_t stream = (cudaStream_t)cuda_stream;
-  // the header and the per-unit counters must start at zero; the rest is written before it is read
-  if (cudaMemsetAsync(ws + w.off_hdr, 0, w.off_part - w.off_hdr, stream) != cudaSuccess)
-    return LAQ_ERR_CUDA;
+  // run_scoring clears the header and the per-unit counters, which must start at zero; the rest
+  // of the scratch is written before it is read
   int launches = 0;
-  st = d.score_raw                  ? score_raw_launch(*p, d, w, q, k, ws, stream, &launches)
-       : (d.D == 128 && d.M <= 256) ? score_tc_launch(*p, d, w, q, k, ws, stream, &launches)
-                                    : score_simt_launch(*p, d, w, q, k, ws, stream, &launches);
-  if (st != LAQ_OK) return st;
-  return pool_launch(d, (const float*)(ws + w.off_colsum), w.L_pad, scores, stream, &launches);
+  st = run_scoring(p, d, w, q, k, ws, stream, &launches);
+  if (st == LAQ_OK)
+    st = pool_launch(d, (const float*)(ws + w.off_colsum), w.L_pad, scores, stream, &launches);
+  set_last_launch_count(launches);
+  return st;
 }

@@ -37,11 +37,6 @@
 #include "laq_internal.cuh"
 #include "softmax_math.cuh"
 
-#ifndef LAQ_PREFETCH_TILES
-#define LAQ_PREFETCH_TILES 0  // 128-key tiles the L2 prefetch of sweep 1 runs ahead of the loads (0 = off:
-                              // measured 4 % slower with 4 tiles, the four-stage ring already covers the latency)
-#endif
-
 #ifndef LAQ_WAIT_HINT_NS
 #define LAQ_WAIT_HINT_NS 2000  // longest hardware suspension of one mbarrier poll
 #endif
@@ -187,13 +182,6 @@ __device__ __forceinline__ void tma_load_5d_hint(uint32_t dst, const CUtensorMap
       "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
       "[%0], [%1, {%3, %4, %5, %6, %7}], [%2], %8;" ::"r"(dst),
       "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "l"(policy)
-      : "memory");
-}
-__device__ __forceinline__ void tma_prefetch_5d(const CUtensorMap* map, int c0, int c1, int c2, int c3,
-                                                int c4, uint64_t policy) {
-  asm volatile(
-      "cp.async.bulk.prefetch.tensor.5d.L2.global.tile.L2::cache_hint [%0, {%1, %2, %3, %4, %5}], %6;" ::"l"(map),
-      "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "l"(policy)
       : "memory");
 }
 // D[tmem] (+)= A[smem] * B[smem]; the two shared-memory descriptors are passed as (low, high) words.
@@ -436,6 +424,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
   constexpr uint32_t kSlotShift = kWide ? 1u : 2u;   // log2 of the K stages = accumulator buffers
   constexpr uint32_t kTbCols = kWide ? 256u : 128u;  // TMEM columns per accumulator buffer
   constexpr int RB = kWide ? 2 : 1;                  // 128-row blocks per tile in sweep 1
+  long long clk0 = 0;
+  unsigned long long ns0 = 0;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    clk0 = clock64();
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns0));
+  }
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   Ctl* ctl = reinterpret_cast<Ctl*>(smem_raw);
   const uint32_t smem_base = smem_u32(smem_raw);
@@ -500,17 +494,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       const uint64_t pol_keep = l2_policy_evict_last(), pol_drop = l2_policy_evict_first();
       unsigned int* ticket_ctr = reinterpret_cast<unsigned int*>(&a.hdr[HDR_TICKET]);
       const Task stop = {-1, 0, 0, 0, 0, 0, 0, 0, 0};
-      // Asks L2 for tiles [first, first+count) of a sweep-1 task ahead of the loads into shared
-      // memory, so that the DRAM latency is not paid inside the shared-memory ring.
-      auto prefetch_tiles = [&](const Task& t, int first, int count) {
-        if (t.sweep != 0) return;
-        const int last = min(t.n_tiles, first + count);
-        for (int i = first; i < last; ++i) {
-          const int key0 = (t.tile0 + i) * TILE_KEYS;
-          tma_prefetch_5d(&tmap_k, 0, key0, t.h, t.b, t.layer, pol_keep);
-          tma_prefetch_5d(&tmap_k, 64, key0, t.h, t.b, t.layer, pol_keep);
-        }
-      };
       int* prefix = ctl->task_prefix;
       if (a.sl.n > 0) {
         int acc = 0;
@@ -525,7 +508,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         const uint32_t t0 = atomicAdd(ticket_ctr, 1u);
         if (t0 < a.total_tickets) decode_ticket(a, prefix, t0, task);
       }
-      if (LAQ_PREFETCH_TILES > 0) prefetch_tiles(task, 0, LAQ_PREFETCH_TILES);
       bool ok = true;
       while (ok) {
         // the next ticket is in flight while this task's loads are issued
@@ -558,7 +540,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         // sweep 1 asks L2 to keep the tile for the second sweep, which then lets it go
         const uint64_t pol = task.sweep == 0 ? pol_keep : pol_drop;
         Task next = stop;
-        bool next_known = false;
         for (int i = 0; i < task.n_tiles; ++i) {
           const uint32_t s = kcount & slot_mask;
           // the stage is free once the MMAs of the tile that used it last have completed
@@ -574,21 +555,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
           tma_load_5d_hint(dst + kKStageBytes / 2, &tmap_k, bar, 64, key0, task.h, task.b, task.layer,
                            pol);
           ++kcount;
-          if (LAQ_PREFETCH_TILES > 0) {
-            // keep the L2 prefetch LAQ_PREFETCH_TILES tiles ahead, across the task boundary
-            const int ahead = i + LAQ_PREFETCH_TILES;
-            if (ahead < task.n_tiles) {
-              prefetch_tiles(task, ahead, 1);
-            } else {
-              if (!next_known) {
-                next_known = true;
-                if (next_ticket < a.total_tickets) decode_ticket(a, prefix, next_ticket, next);
-              }
-              prefetch_tiles(next, ahead - task.n_tiles, 1);
-            }
-          }
         }
-        if (!next_known && next_ticket < a.total_tickets) decode_ticket(a, prefix, next_ticket, next);
+        if (next_ticket < a.total_tickets) decode_ticket(a, prefix, next_ticket, next);
         task = next;
       }
       if (ctl->abort) {
@@ -900,6 +868,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
   // ---- teardown
   tc_fence_before();
   __syncthreads();
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    unsigned long long ns1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns1));
+    *reinterpret_cast<long long*>(&a.hdr[HDR_CYCLES]) = clock64() - clk0;
+    *reinterpret_cast<long long*>(&a.hdr[HDR_NANOS]) = (long long)(ns1 - ns0);
+  }
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
@@ -915,17 +889,16 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
+  // looked up once; a function-local static is initialised exactly once even with several host threads
+  static const EncodeTiledFn fn = [] {
     void* sym = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) ==
             cudaSuccess &&
         qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(sym);
-  }
+      return reinterpret_cast<EncodeTiledFn>(sym);
+    return static_cast<EncodeTiledFn>(nullptr);
+  }();
   return fn;
 }
 

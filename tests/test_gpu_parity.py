@@ -543,11 +543,19 @@ def test_config1_full_with_planted_key(laq):
 
 
 def sampled_parity(laq, cfg, budgets, units, device="cuda"):
-    """Runs the full-size problem on the GPU and checks the listed units against the oracle."""
+    """Runs the full-size problem on the GPU, in the launch configuration the benchmark times, and
+    checks the listed units against the oracle. The scores do not depend on the budget, so the
+    oracle scores every sampled unit once (all of them in one call, spread over its OpenMP
+    threads) and only re-selects per budget."""
     inp = synth.make_inputs(cfg, device)
     q, k, v = inp["q"], inp["k"], inp["v"]
     R, L, D = cfg.keep_tail, cfg.prompt_len, cfg.head_dim
     NL, Bt, Hkv = cfg.n_layers, cfg.batch, cfg.n_kv_heads
+    units = sorted(set(int(u) for u in units))
+    slices = [synth.unit_slices(cfg, inp, u) for u in units]
+    qs = torch.stack([x[0][0] for x in slices])   # [n, 1, G, W, D]
+    ks = torch.stack([x[1][0] for x in slices])   # [n, 1, 1, L, D]
+    ref_scores = orc.evict(qs, ks, None, R, cfg.pool_kernel, max(budgets), want_idx=False)["scores"]
     worst = 0.0
     ws = None
     for B in budgets:
@@ -565,16 +573,17 @@ def sampled_parity(laq, cfg, budgets, units, device="cuda"):
         laq.laq_evict(p, q, k, v, k_out, v_out, idx2, scores2, ws)
         assert torch.equal(scores, scores2) and torch.equal(idx, idx2)
         del scores2, idx2
-        for u in units:
+        for j, u in enumerate(units):
             h, b, n = u % Hkv, (u // Hkv) % Bt, u // (Hkv * Bt)
-            qu, ku, vu = synth.unit_slices(cfg, inp, u)
-            ref = orc.evict(qu, ku, vu, R, cfg.pool_kernel, B)
+            ku, vu = slices[j][1], slices[j][2]
+            ref_s = ref_scores[j, 0, 0]
+            ref_idx = orc.select(ref_s, L, R, B, sorted_variant=True)
             got_s = scores[n, b, h].cpu().numpy()
-            err = score_rel_err(got_s, ref["scores"][0, 0, 0])
+            err = score_rel_err(got_s, ref_s)
             worst = max(worst, err)
             assert err <= SCORE_RTOL, f"unit {u} B {B}: score rel err {err:.3e}"
             gi = idx[n, b, h].cpu().numpy()
-            check_index_set(gi, ref["idx"][0, 0, 0], ref["scores"][0, 0, 0], L, R, B)
+            check_index_set(gi, ref_idx, ref_s, L, R, B)
             assert (gi == orc.select(got_s, L, R, B, sorted_variant=True)).all()
             assert (bits(k_out[n, b, h]) == bits(ku[0, 0, 0])[gi]).all()
             assert (bits(v_out[n, b, h]) == bits(vu[0, 0, 0])[gi]).all()
@@ -585,24 +594,38 @@ def sampled_parity(laq, cfg, budgets, units, device="cuda"):
     return worst
 
 
+def spread_units(cfg, n_random):
+    """First and last layer, every batch item and KV head at least once, plus seeded random units."""
+    Hkv, Bt, NL = cfg.n_kv_heads, cfg.batch, cfg.n_layers
+    units = set(synth.sample_units(cfg, n_random))
+    for b in range(Bt):  # every batch item, in the first and in the last layer, rotating the head
+        units.add((0 * Bt + b) * Hkv + b % Hkv)
+        units.add(((NL - 1) * Bt + b) * Hkv + (b + 1) % Hkv)
+    units.add(cfg.units - 1)
+    return sorted(units)
+
+
 def test_config2_full_size_sampled_units(laq):
     cfg = synth.CONFIGS[2]
-    sampled_parity(laq, cfg, cfg.budgets, synth.sample_units(cfg, 4))
+    sampled_parity(laq, cfg, cfg.budgets, spread_units(cfg, 8))
 
 
 def test_config3_full_size_sampled_units(laq):
     cfg = synth.CONFIGS[3]
-    units = [0, 5, cfg.units // 2 + 3, cfg.units - 1]
-    sampled_parity(laq, cfg, (128, 2048), units)
+    units = spread_units(cfg, 6)
+    assert len(units) >= 16
+    sampled_parity(laq, cfg, cfg.budgets, units)   # 128, 256, 512, 1024, 2048
 
 
 def test_config4_full_size_sampled_units(laq):
     cfg = synth.CONFIGS[4]
-    units = [0, 777, cfg.units - 1]
+    units = spread_units(cfg, 4)
+    assert len(units) >= 16
     sampled_parity(laq, cfg, cfg.budgets, units)
 
 
 def test_config5_full_size_one_pool(laq):
     cfg = synth.CONFIGS[5]
-    units = [1, cfg.units - 1]  # the last unit's keys lie beyond 2^32 bytes from the base
-    sampled_parity(laq, cfg, (2048,), units)
+    units = spread_units(cfg, 4)  # the last unit's keys lie beyond 2^32 bytes from the base
+    assert len(units) >= 16 and units[-1] == cfg.units - 1
+    sampled_parity(laq, cfg, cfg.budgets, units)   # 256 and 2048
