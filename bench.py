@@ -345,6 +345,9 @@ def main():
         total_ms = start.elapsed_time(stop)
     if laq.laq_last_device_status(p, ws) != laq.LAQ_OK:
         raise RuntimeError("laq_evict reported a device-side error")
+    # what the scoring kernel of the last step recorded about itself: SM cycles and wall time of
+    # its first block, i.e. the SM clock it really ran at (the board lowers it under load)
+    kernel_cycles, kernel_ns = laq.laq_last_kernel_clock(ws)
     from paper_2505_20334_b200 import multi
 
     total_ms = multi.max_over_ranks(total_ms, dev)
@@ -363,6 +366,12 @@ def main():
                 "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
                 "peak_source": peak_src, "algorithmic_bytes_per_launch": score_bytes,
                 "kernel_ms": score_ms, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
+    if kernel_ns > 0 and not raw:
+        sms_ = torch.cuda.get_device_properties(dev).multi_processor_count
+        tile_sweeps = 2.0 * NL * Hkv * sum(-(-x // 128) for x in (lens or [L] * Bt)) / sms_
+        roofline["in_kernel"] = {"sm_mhz": kernel_cycles / kernel_ns * 1e3, "sm_cycles": kernel_cycles,
+                                 "cycles_per_128key_tile_and_sweep_per_sm": kernel_cycles / tile_sweeps,
+                                 "source": "clock64 / globaltimer of the kernel's first block, last step"}
     # The scoring kernel's busiest unit is the MUFU: two base-2 exponentials per (row, key) pair
     # (one per sweep) at 16 per clock and SM.
     n_exp = 2.0 * NL * Hkv * cfg.rows * tokens_per_step

