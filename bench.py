@@ -11,14 +11,19 @@ long-context cache (32 layers, 32/8 heads, batch 4, L = 32768, W = 32, pool kern
   cpu_baseline the fp64 CPU oracle timed on this machine's cores on a sample of the same units
 
 ``--impl reference`` times the CPU oracle instead (it is the only reference this method has).
-With N > 1 GPUs (torchrun) every rank evicts its own copy of the workload: the units are
-independent, so there is no data-path collective; only the timing is reduced over ranks.
+With ``--gpus N`` (N > 1) the script starts N ranks itself, one per GPU, through
+``torch.distributed.run`` (or runs as one of them when a launcher has already set WORLD_SIZE).
+The units are independent, so there is no data-path collective; only the timing is reduced over
+ranks. ``--scaling weak`` (default): every rank evicts its own cache of the full size;
+``--scaling strong``: the layers of one cache are split over the ranks.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -61,7 +66,54 @@ def parse_args():
                     help="time the steps as replays of one captured CUDA graph (launch-bound small workloads)")
     ap.add_argument("--tiles-per-task", type=int, default=0)
     ap.add_argument("--lag-tasks", type=int, default=0)
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="N > 1: weak = one full-size cache per rank, strong = one cache's layers split over the ranks")
+    ap.add_argument("--stub-step", action="store_true",
+                    help="host-logic check of the multi-rank path without a GPU: gloo backend, the step is a "
+                         "timed sleep (used by the CPU tests; the line it prints is not a measurement)")
     return ap.parse_args()
+
+
+def spawn_ranks(args) -> int:
+    """--gpus N without a launcher: re-run this script as N ranks of one node."""
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+           f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1", "--master-port", str(port),
+           os.path.abspath(__file__), *sys.argv[1:]]
+    return subprocess.call(cmd)
+
+
+def run_stub(args):
+    """The multi-rank plumbing of main() on CPU: process group, barrier, per-rank shard, MAX over
+    ranks of the step time, one JSON line from rank 0."""
+    import torch.distributed as dist
+    from paper_2505_20334_b200 import multi, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    cfg = workload(args)
+    layers = multi.shard_units(cfg.n_layers, world, rank) if args.scaling == "strong" else (0, cfg.n_layers)
+    tokens = cfg.batch * cfg.prompt_len
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time.sleep(0.002 * (rank + 1))  # the last rank is the slow one
+    my_ms = (time.perf_counter() - t0) * 1e3 / max(1, args.steps)
+    ms = multi.max_over_ranks(my_ms)
+    if world > 1:
+        dist.barrier()
+    if rank == 0:
+        per_step = tokens * world if args.scaling == "weak" else tokens
+        print(json.dumps({"metric": METRIC, "value": per_step / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+                          "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                          "higher_is_better": True, "scaling": args.scaling, "stub": True,
+                          "layers_of_rank0": list(layers), "config": config_dict(cfg, args.budget, args)}))
+    if world > 1:
+        dist.destroy_process_group()
 
 
 def measured_peaks():
@@ -195,6 +247,9 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    if "WORLD_SIZE" in os.environ:
+        # a launcher pins every rank to one OpenMP thread; here rank 0 alone works, on all host cores
+        os.environ["OMP_NUM_THREADS"] = str(os.cpu_count() or 1)
     import torch
     from oracle import laq_oracle as orc
     from paper_2505_20334_b200 import synth
@@ -227,15 +282,18 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": config_dict(cfg, B),
+        "data": "synthetic", "config": config_dict(cfg, B, args),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": int(threads), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
 
-def config_dict(cfg, B):
-    return {"workload": f"config {cfg.cfg_id}: {cfg.name}", "n_layers": cfg.n_layers,
+def config_dict(cfg, B, args, lens=None):
+    """The workload and every option that changes it; the same keys in both arms."""
+    return {"workload": f"config {cfg.cfg_id}: {cfg.name}", "score_mode": args.score_mode,
+            "pool_mode": args.pool_mode, "local_window": args.local_window, "seq_lens": lens,
+            "cuda_graph": bool(args.graph), "n_layers": cfg.n_layers,
             "batch": cfg.batch, "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads,
             "head_dim": cfg.head_dim, "prompt_len": cfg.prompt_len, "window_len": cfg.window_len,
             "keep_tail": cfg.keep_tail, "pool_kernel": cfg.pool_kernel, "budget": B,
@@ -245,8 +303,13 @@ def config_dict(cfg, B):
 
 def main():
     args = parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.stub_step:
+        run_stub(args)
         return
 
     import torch
@@ -265,10 +328,16 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
         dist.barrier()
     from paper_2505_20334_b200 import binding as laq
-    from paper_2505_20334_b200 import synth
+    from paper_2505_20334_b200 import multi, synth
 
-    cfg = workload(args)
-    if world > 1:
+    cfg_full = cfg = workload(args)
+    if world > 1 and args.scaling == "strong":
+        # one cache, its layers split over the ranks (units are independent: no exchange)
+        lo, hi = multi.shard_units(cfg.n_layers, world, rank)
+        if hi <= lo:
+            raise SystemExit("--scaling strong needs at least one layer per rank")
+        cfg = cfg.scaled(n_layers=hi - lo, cfg_id=cfg.cfg_id + 1000 * rank)
+    elif world > 1:
         cfg = cfg.scaled(cfg_id=cfg.cfg_id + 1000 * rank)  # every rank draws its own cache
     B = args.budget
     inputs = synth.make_inputs(cfg, dev)
@@ -348,11 +417,12 @@ def main():
     # what the scoring kernel of the last step recorded about itself: SM cycles and wall time of
     # its first block, i.e. the SM clock it really ran at (the board lowers it under load)
     kernel_cycles, kernel_ns = laq.laq_last_kernel_clock(ws)
-    from paper_2505_20334_b200 import multi
-
     total_ms = multi.max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / K
-    value = multi.whole_job_tokens_per_s(tokens_per_step, world, ms_per_step)
+    # weak: every rank evicts tokens_per_step prompt tokens (all layers); strong: the ranks share
+    # the layers of one cache, so the job as a whole evicts tokens_per_step per step
+    value = multi.whole_job_tokens_per_s(tokens_per_step, world if args.scaling == "weak" else 1,
+                                         ms_per_step)
 
     peak, peak_src = measured_peaks()
     score_bytes, gather_bytes = algorithmic_bytes(cfg, B, tokens_per_step / Bt)
@@ -425,11 +495,11 @@ def main():
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "scaling": args.scaling, "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
-            "config": dict(config_dict(cfg, B), score_mode=args.score_mode, pool_mode=args.pool_mode,
-                           local_window=args.local_window, seq_lens=lens, cuda_graph=args.graph),
-            "kv_entries_per_s": NL * Hkv * tokens_per_step * world / (ms_per_step * 1e-3),
+            "config": config_dict(cfg_full, B, args, lens),
+            "kv_entries_per_s": cfg_full.n_layers * Hkv * tokens_per_step *
+                                (world if args.scaling == "weak" else 1) / (ms_per_step * 1e-3),
             "roofline": roofline, "step_roofline": step_roofline, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": launches_per_step * K, "clocks": clocks,
         }))

@@ -1,7 +1,10 @@
 """The multi-GPU plumbing (no data-path collective: shard the independent units, reduce only the
 timing) exercised with two gloo ranks on CPU."""
+import json
 import os
 import socket
+import subprocess
+import sys
 
 import pytest
 import torch
@@ -62,3 +65,22 @@ def test_two_gloo_ranks_reduce_timing_and_cover_all_units():
 
 def test_max_over_ranks_without_process_group_is_identity():
     assert multi.max_over_ranks(2.5) == 2.5
+
+
+def test_bench_gpus_flag_starts_that_many_ranks():
+    """`bench.py --gpus 2` with no launcher around it must start two ranks itself and report
+    n_gpus 2 with the slowest rank's time (stubbed step on CPU: gloo, no GPU work)."""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items()
+           if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--stub-step",
+                          "--steps", "3", "--scaling", "strong"], capture_output=True, text=True,
+                         env=env, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1  # rank 0 alone prints
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["scaling"] == "strong"
+    assert line["ms_per_step"] >= 3.9  # rank 1 sleeps 4 ms per step: the maximum over ranks
+    assert line["layers_of_rank0"] == [0, 16]
+    assert line["config"]["workload"].startswith("config 3")
