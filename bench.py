@@ -54,6 +54,8 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling)")
     ap.add_argument("--prompt-len", type=int, default=0, help="override the prompt length (profiling)")
+    ap.add_argument("--window", type=int, default=0,
+                    help="override W, the lookahead queries per head (Section 6.2 ablates 1, 2 and 8 steps)")
     ap.add_argument("--local-window", type=int, default=0,
                     help="LAQ++ (Eq. 5): this many of the window's queries are causal local queries")
     ap.add_argument("--score-mode", default="softmax", choices=["softmax", "raw"],
@@ -203,6 +205,8 @@ def workload(args):
         cfg = cfg.scaled(batch=args.batch)
     if args.prompt_len:
         cfg = cfg.scaled(prompt_len=args.prompt_len)
+    if args.window:
+        cfg = cfg.scaled(window_len=args.window)  # the retained tail keeps its size
     return cfg
 
 
@@ -429,7 +433,7 @@ def main():
     achieved = score_bytes / (score_ms * 1e-3) / 1e9
     raw = args.score_mode == "raw"
     # the ncu figures were taken on the full headline workload only
-    captured = args.config == 3 and not (args.layers or args.batch or args.prompt_len or lens)
+    captured = args.config == 3 and not (args.layers or args.batch or args.prompt_len or lens or args.window)
     traffic = (NCU_TRAFFIC_BYTES_RAW if raw else NCU_TRAFFIC_BYTES) if captured else None
     roofline = {"bound": "hbm", "kernel": "score_raw_d128_kernel" if raw else "score_tc_kernel",
                 "achieved": achieved, "peak": peak,

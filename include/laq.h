@@ -136,6 +136,7 @@ typedef struct {
 } laq_params;
 
 #define LAQ_MAX_RAGGED_BATCH 512
+#define LAQ_MAX_LAYER_BUDGETS 256
 
 /* Fills the stride fields of `p` for densely packed tensors in the index order shown above. */
 LAQ_API void laq_params_dense_strides(laq_params* p);
@@ -220,6 +221,42 @@ LAQ_API laq_status laq_compact(const laq_params* p, const void* k, const void* v
 LAQ_API laq_status laq_evict(const laq_params* p, const void* q, const void* k, const void* v,
                      void* k_out, void* v_out, int32_t* idx, float* scores, void* ws,
                      size_t ws_bytes, void* cuda_stream);
+
+/*
+ * laq_evict with one budget per layer. The paper evicts to a fixed budget (Section 5.2) and names
+ * layer-wise budgets of the PyramidKV kind as a combination it is compatible with (Section 5.1);
+ * the units of different layers are independent, so only steps 5 and 6 change.
+ *   layer_budgets  HOST, int32 [NL], read during the call only: layer n keeps layer_budgets[n]
+ *                  positions per (batch, KV head), R < layer_budgets[n] < L (and below every
+ *                  seq_lens entry). p->budget must equal the largest of them (it sizes the
+ *                  workspace). NL <= LAQ_MAX_LAYER_BUDGETS.
+ *   idx            optional, device int32: ONE ragged pool, layer after layer; layer n holds
+ *                  [Bt][Hkv][layer_budgets[n]] entries and starts at entry
+ *                  Bt*Hkv*(layer_budgets[0] + ... + layer_budgets[n-1])
+ *   k_out, v_out   device bf16, the same ragged pool with D elements per entry (densely packed:
+ *                  the o_stride_* fields are not used); either may be NULL
+ *   scores         optional, device fp32, dense [NL][Bt][Hkv][L-R] as for laq_evict
+ * laq_layers_pool_entries() returns the number of entries of the pool (0 for invalid arguments).
+ * Errors: as laq_evict, LAQ_ERR_UNSUPPORTED for more than LAQ_MAX_LAYER_BUDGETS layers.
+ */
+LAQ_API size_t laq_layers_pool_entries(const laq_params* p, const int32_t* layer_budgets);
+LAQ_API laq_status laq_evict_layers(const laq_params* p, const int32_t* layer_budgets, const void* q,
+                                    const void* k, const void* v, void* k_out, void* v_out,
+                                    int32_t* idx, float* scores, void* ws, size_t ws_bytes,
+                                    void* cuda_stream);
+
+/*
+ * The keep-set of a StreamingLLM-style cache: the first n_sink positions ("attention sinks") and
+ * the most recent budget - n_sink positions of every prompt. Section 4.2 starts the lookahead from
+ * a low-budget cache of this kind (or of the SnapKV kind, which is laq_evict with
+ * local_window = window_len); feeding these indices to laq_compact builds it.
+ *   idx   device, int32, dense [NL][Bt][Hkv][B], ascending: 0 .. n_sink-1, then Lb-(B-n_sink) .. Lb-1
+ *         (Lb = seq_lens[b] if given, else L)
+ * Only n_layers, batch, n_kv_heads, prompt_len, budget and seq_lens of `p` are read.
+ * Errors: LAQ_ERR_INVALID_ARG (n_sink outside [0, B], B >= Lb), LAQ_ERR_CUDA.
+ */
+LAQ_API laq_status laq_streaming_indices(const laq_params* p, int32_t n_sink, int32_t* idx,
+                                         void* cuda_stream);
 
 /*
  * Recall of one selection against another (Section 3, Eq. 1-3):

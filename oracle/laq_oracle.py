@@ -184,3 +184,33 @@ def evict(q, k, v, R, kernel, B, scale=None, units=None, want_colsum=False, fast
     if want_colsum:
         out["colsum"] = colsum
     return out
+
+
+def evict_layers(q, k, v, R, kernel, budgets, **kw):
+    """One budget per layer (layer-wise budgets, Sections 5.1-5.2): layer n is evicted on its own
+    with budgets[n], and the results are laid end to end in one ragged pool, layer after layer,
+    each layer as [Bt][Hkv][budgets[n]] entries. Returns {'idx' [entries] int32, 'k_out', 'v_out'
+    [entries][D] uint16, 'scores' [NL,Bt,Hkv,L-R]}. Keyword arguments as for evict()."""
+    q, k = _bits(q), _bits(k)
+    v = None if v is None else _bits(v)
+    NL = q.shape[0]
+    assert len(budgets) == NL
+    idx, k_out, v_out, scores = [], [], [], []
+    for n in range(NL):
+        r = evict(q[n:n + 1], k[n:n + 1], None if v is None else v[n:n + 1], R, kernel, int(budgets[n]), **kw)
+        idx.append(r["idx"].reshape(-1))
+        k_out.append(r["k_out"].reshape(-1, k.shape[-1]))
+        if v is not None:
+            v_out.append(r["v_out"].reshape(-1, k.shape[-1]))
+        scores.append(r["scores"])
+    return {"idx": np.concatenate(idx), "k_out": np.concatenate(k_out),
+            "v_out": np.concatenate(v_out) if v is not None else None,
+            "scores": np.concatenate(scores)}
+
+
+def streaming_indices(L, B, n_sink, seq_len=None):
+    """The keep-set of a StreamingLLM-style cache for one prompt, as the literal list: the first
+    n_sink positions and the last B - n_sink positions of the prompt's Lb = seq_len or L."""
+    Lb = L if seq_len is None else int(seq_len)
+    assert 0 <= n_sink <= B < Lb <= L
+    return np.array(list(range(n_sink)) + list(range(Lb - (B - n_sink), Lb)), np.int32)

@@ -29,7 +29,8 @@ EXPORTS = (
     "laq_params_dense_strides", "laq_workspace_bytes", "laq_score", "laq_select", "laq_compact",
     "laq_evict", "laq_last_device_status", "laq_last_launch_count", "laq_status_string",
     "laq_version", "laq_set_stage_events", "laq_host_staging_bytes", "laq_evict_host",
-    "laq_score_static", "laq_recall", "laq_last_kernel_clock",
+    "laq_score_static", "laq_recall", "laq_last_kernel_clock", "laq_evict_layers",
+    "laq_layers_pool_entries", "laq_streaming_indices",
 )
 
 
@@ -102,6 +103,13 @@ def _load() -> ctypes.CDLL:
     lib.laq_last_kernel_clock.argtypes = [vp, sz, vp, ctypes.POINTER(ctypes.c_int64),
                                           ctypes.POINTER(ctypes.c_int64)]
     lib.laq_last_kernel_clock.restype = ctypes.c_int
+    i32p = ctypes.POINTER(ctypes.c_int32)
+    lib.laq_evict_layers.argtypes = [pp, i32p, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.laq_evict_layers.restype = ctypes.c_int
+    lib.laq_layers_pool_entries.argtypes = [pp, i32p]
+    lib.laq_layers_pool_entries.restype = sz
+    lib.laq_streaming_indices.argtypes = [pp, ctypes.c_int32, vp, vp]
+    lib.laq_streaming_indices.restype = ctypes.c_int
     lib.laq_version.argtypes = []
     lib.laq_version.restype = ctypes.c_int
     return lib
@@ -295,27 +303,64 @@ def evict(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, budget: int, pool_k
 
 
 
+def _budget_array(budgets):
+    return (ctypes.c_int32 * len(budgets))(*[int(b) for b in budgets])
+
+
+def laq_layers_pool_entries(p: LaqParams, budgets) -> int:
+    return int(lib.laq_layers_pool_entries(ctypes.byref(p), _budget_array(budgets)))
+
+
+def laq_evict_layers(p: LaqParams, budgets, q, k, v, k_out, v_out, idx, scores, ws, stream=None,
+                     check=True) -> int:
+    """``laq_evict`` with one budget per layer; idx / k_out / v_out are one ragged pool (laq.h)."""
+    wp, wn = _ws_args(ws)
+    st = lib.laq_evict_layers(ctypes.byref(p), _budget_array(budgets), _ptr(q), _ptr(k), _ptr(v),
+                              _ptr(k_out), _ptr(v_out), _ptr(idx), _ptr(scores), wp, wn, _stream(stream))
+    if check and st != LAQ_OK:
+        raise LaqError(st, "laq_evict_layers")
+    return st
+
+
+def laq_streaming_indices(p: LaqParams, n_sink: int, idx, stream=None, check=True) -> int:
+    st = lib.laq_streaming_indices(ctypes.byref(p), int(n_sink), _ptr(idx), _stream(stream))
+    if check and st != LAQ_OK:
+        raise LaqError(st, "laq_streaming_indices")
+    return st
+
+
 def evict_layer_budgets(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, budgets, pool_kernel: int = 7,
-                        keep_tail: Optional[int] = None, local_window: int = 0, stream=None):
+                        keep_tail: Optional[int] = None, local_window: int = 0, stream=None,
+                        seq_lens=None):
     """Eviction with one budget per layer (the paper fixes the budget, Section 5.2, and names
-    layer-wise budgets such as PyramidKV's as a combination). The units of different layers are
-    independent, so this is one ``laq_evict`` call per run of layers that share a budget, on layer
-    slices of the same tensors (no copies). Returns a list with one dict per layer
-    ('k_out', 'v_out' [Bt,Hkv,B_l,D], 'idx' [Bt,Hkv,B_l])."""
-    NL = q.shape[0]
+    layer-wise budgets such as PyramidKV's as a combination): one ``laq_evict_layers`` call that
+    writes the compressed caches of all layers into one ragged pool. Returns the pool tensors and a
+    list with one dict of views per layer ('k_out', 'v_out' [Bt,Hkv,B_l,D], 'idx' [Bt,Hkv,B_l])."""
+    NL, Bt, Hq, W, D = q.shape
+    Hkv = k.shape[2]
     if len(budgets) != NL:
         raise ValueError("evict_layer_budgets: one budget per layer is required")
-    out, ws, lo = [None] * NL, None, 0
-    while lo < NL:
-        hi = lo + 1
-        while hi < NL and budgets[hi] == budgets[lo]:
-            hi += 1
-        r = evict(q[lo:hi], k[lo:hi], v[lo:hi], int(budgets[lo]), pool_kernel=pool_kernel,
-                  keep_tail=keep_tail, stream=stream, local_window=local_window)
-        for n in range(lo, hi):
-            out[n] = {"k_out": r["k_out"][n - lo], "v_out": r["v_out"][n - lo], "idx": r["idx"][n - lo]}
-        lo = hi
-    return out
+    R = W if keep_tail is None else keep_tail
+    p = params_for(q, k, R, pool_kernel, max(int(b) for b in budgets), v=v)
+    p.local_window = local_window
+    p.set_seq_lens(seq_lens)
+    entries = laq_layers_pool_entries(p, budgets)
+    if entries == 0:
+        raise LaqError(LAQ_ERR_INVALID_ARG, "laq_layers_pool_entries")
+    idx = torch.empty(entries, dtype=torch.int32, device=k.device)
+    k_out = torch.empty((entries, D), dtype=k.dtype, device=k.device)
+    v_out = torch.empty_like(k_out)
+    ws = alloc_workspace(p, k.device)
+    laq_evict_layers(p, budgets, q, k, v, k_out, v_out, idx, None, ws, stream)
+    layers, row = [], 0
+    for n in range(NL):
+        B = int(budgets[n])
+        cnt = Bt * Hkv * B
+        layers.append({"k_out": k_out[row:row + cnt].view(Bt, Hkv, B, D),
+                       "v_out": v_out[row:row + cnt].view(Bt, Hkv, B, D),
+                       "idx": idx[row:row + cnt].view(Bt, Hkv, B)})
+        row += cnt
+    return {"idx": idx, "k_out": k_out, "v_out": v_out, "layers": layers, "params": p, "ws": ws}
 
 
 def laq_host_staging_bytes(p: LaqParams) -> int:

@@ -64,6 +64,7 @@ laq_status derive_dims(const laq_params* p, Dims* d) {
   d->tiles_per_task = p->tiles_per_task;
   d->sched_lag_tasks = p->sched_lag_tasks;
   d->scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / sqrtf((float)d->D);
+  d->lb.n = 0;
   return derive_seq_lens(p, &d->sl);
 }
 
@@ -258,13 +259,11 @@ laq_status laq_compact(const laq_params* p, const void* k, const void* v, const 
   return st;
 }
 
-laq_status laq_evict(const laq_params* p, const void* q, const void* k, const void* v,
-                     void* k_out, void* v_out, int32_t* idx, float* scores, void* ws,
-                     size_t ws_bytes, void* cuda_stream) {
-  g_last_launches = 0;
-  Dims d;
-  laq_status st = derive_dims(p, &d);
-  if (st != LAQ_OK) return st;
+// Steps 1-6 for validated sizes `d` (d.lb may hold per-layer budgets).
+static laq_status evict_impl(const laq_params* p, const Dims& d, const void* q, const void* k,
+                             const void* v, void* k_out, void* v_out, int32_t* idx, float* scores,
+                             void* ws, size_t ws_bytes, void* cuda_stream) {
+  laq_status st;
   if (!q || !k || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) ||
       !aligned16(v_out))
     return LAQ_ERR_INVALID_ARG;
@@ -297,6 +296,77 @@ laq_status laq_evict(const laq_params* p, const void* q, const void* k, const vo
     st = compact_launch(*p, d, k, v, idx_dev, k_out, v_out, stream, &launches);
   g_last_launches = launches;
   return st;
+}
+
+laq_status laq_evict(const laq_params* p, const void* q, const void* k, const void* v,
+                     void* k_out, void* v_out, int32_t* idx, float* scores, void* ws,
+                     size_t ws_bytes, void* cuda_stream) {
+  g_last_launches = 0;
+  Dims d;
+  const laq_status st = derive_dims(p, &d);
+  if (st != LAQ_OK) return st;
+  return evict_impl(p, d, q, k, v, k_out, v_out, idx, scores, ws, ws_bytes, cuda_stream);
+}
+
+// Validates the per-layer budgets against `d` (whose B must be the largest) and fills d->lb.
+static laq_status derive_layer_budgets(const laq_params* p, const int32_t* layer_budgets, Dims* d) {
+  if (!layer_budgets) return LAQ_ERR_INVALID_ARG;
+  if (d->NL > LAQ_MAX_LAYER_BUDGETS) return LAQ_ERR_UNSUPPORTED;
+  int largest = 0;
+  int64_t row = 0;
+  for (int n = 0; n < d->NL; ++n) {
+    const int32_t B = layer_budgets[n];
+    if (B <= d->R || B >= d->L) return LAQ_ERR_INVALID_ARG;
+    for (int b = 0; b < d->sl.n; ++b)
+      if (B >= d->sl.len[b]) return LAQ_ERR_INVALID_ARG;
+    d->lb.B[n] = B;
+    d->lb.row0[n] = row;
+    row += (int64_t)d->Bt * d->Hkv * B;
+    if (B > largest) largest = B;
+  }
+  if (largest != p->budget) return LAQ_ERR_INVALID_ARG;
+  d->lb.n = d->NL;
+  return LAQ_OK;
+}
+
+size_t laq_layers_pool_entries(const laq_params* p, const int32_t* layer_budgets) {
+  Dims d;
+  if (derive_dims(p, &d) != LAQ_OK || derive_layer_budgets(p, layer_budgets, &d) != LAQ_OK) return 0;
+  return (size_t)(d.lb.row0[d.NL - 1] + (int64_t)d.Bt * d.Hkv * d.lb.B[d.NL - 1]);
+}
+
+laq_status laq_evict_layers(const laq_params* p, const int32_t* layer_budgets, const void* q,
+                            const void* k, const void* v, void* k_out, void* v_out, int32_t* idx,
+                            float* scores, void* ws, size_t ws_bytes, void* cuda_stream) {
+  g_last_launches = 0;
+  Dims d;
+  laq_status st = derive_dims(p, &d);
+  if (st != LAQ_OK) return st;
+  if ((st = derive_layer_budgets(p, layer_budgets, &d)) != LAQ_OK) return st;
+  return evict_impl(p, d, q, k, v, k_out, v_out, idx, scores, ws, ws_bytes, cuda_stream);
+}
+
+laq_status laq_streaming_indices(const laq_params* p, int32_t n_sink, int32_t* idx,
+                                 void* cuda_stream) {
+  g_last_launches = 0;
+  if (!p || !idx || (reinterpret_cast<uintptr_t>(idx) & 3u)) return LAQ_ERR_INVALID_ARG;
+  if (p->n_layers < 1 || p->batch < 1 || p->n_kv_heads < 1 || p->prompt_len < 1 || p->budget < 1 ||
+      p->budget >= p->prompt_len || n_sink < 0 || n_sink > p->budget)
+    return LAQ_ERR_INVALID_ARG;
+  Dims d;
+  memset(&d, 0, sizeof d);
+  d.NL = p->n_layers;
+  d.Bt = p->batch;
+  d.Hkv = p->n_kv_heads;
+  d.L = p->prompt_len;
+  d.B = p->budget;
+  d.U = (int64_t)d.NL * d.Bt * d.Hkv;
+  const laq_status st = derive_seq_lens(p, &d.sl);  // budget < seq_lens[b] <= L
+  if (st != LAQ_OK) return st;
+  int launches = 0;
+  const laq_status st2 = streaming_launch(d, n_sink, idx, (cudaStream_t)cuda_stream, &launches);
+  g_last_launches = launches;
+  return st2;
 }
 
 struct HostStaging {

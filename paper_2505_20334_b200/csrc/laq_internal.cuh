@@ -18,6 +18,26 @@ __host__ __device__ __forceinline__ int unit_len(const SeqLens& sl, int b, int L
   return sl.n > 0 ? sl.len[b] : L;
 }
 
+// One budget per layer (laq_evict_layers), passed to the kernels by value (n = 0: the same budget
+// B for every layer). The outputs of all layers then share one ragged pool: layer n holds
+// Bt*Hkv rows of B[n] entries each, starting at entry row0[n] = Bt*Hkv * (B[0] + ... + B[n-1]).
+struct LayerBudgets {
+  int n;
+  int32_t B[LAQ_MAX_LAYER_BUDGETS];
+  int64_t row0[LAQ_MAX_LAYER_BUDGETS];
+};
+// Budget of unit u and the first entry of its row in the index / output pool.
+__host__ __device__ __forceinline__ int unit_budget(const LayerBudgets& lb, int64_t u,
+                                                    int units_per_layer, int B) {
+  return lb.n > 0 ? lb.B[u / units_per_layer] : B;
+}
+__host__ __device__ __forceinline__ int64_t unit_out_row(const LayerBudgets& lb, int64_t u,
+                                                         int units_per_layer, int B) {
+  if (lb.n == 0) return u * (int64_t)B;
+  const int64_t layer = u / units_per_layer;
+  return lb.row0[layer] + (u % units_per_layer) * (int64_t)lb.B[layer];
+}
+
 // Problem sizes derived from laq_params (notation of laq.h).
 struct Dims {
   int NL, Bt, Hq, Hkv, G, D, L, W, R, kpool, B;
@@ -30,6 +50,7 @@ struct Dims {
   float scale;  // softmax scale
   int tiles_per_task, sched_lag_tasks;  // caller's scheduling knobs (0 = automatic)
   SeqLens sl;   // per-prompt lengths (n = 0: uniform)
+  LayerBudgets lb;  // per-layer budgets (n = 0: B for every layer; otherwise B = the largest)
 };
 
 // Workspace layout (all offsets in bytes from the 256-byte aligned base).
@@ -94,6 +115,10 @@ laq_status pool_select_launch(const Dims& d, const float* colsum, int L_pad, flo
 laq_status compact_launch(const laq_params& p, const Dims& d, const void* k, const void* v,
                           const int32_t* idx, void* k_out, void* v_out, cudaStream_t stream,
                           int* launches);
+
+// StreamingLLM-style keep-set: positions 0..n_sink-1 and the last B - n_sink of every prompt.
+laq_status streaming_launch(const Dims& d, int n_sink, int32_t* idx, cudaStream_t stream,
+                            int* launches);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

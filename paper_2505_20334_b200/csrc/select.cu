@@ -12,11 +12,19 @@ constexpr int kSelWarps = kSelThreads / 32;
 // Geometry shared by the kernels below. Ls_full = L - R is the row length of the score tensor;
 // a unit whose prompt is shorter (per-prompt lengths) scores only its first Lb - R positions.
 struct SelGeom {
-  int Ls_full, Kb, R, B, Bt, Hkv;
+  int Ls_full, R, B, Bt, Hkv;
   SeqLens sl;
+  LayerBudgets lb;
 };
 __device__ __forceinline__ int unit_scored(const SelGeom& g, int64_t u) {
   return unit_len(g.sl, (int)((u / g.Hkv) % g.Bt), g.Ls_full + g.R) - g.R;
+}
+// Slots unit u selects (its budget without the tail) and where its row of kept positions starts.
+__device__ __forceinline__ int unit_kb(const SelGeom& g, int64_t u) {
+  return unit_budget(g.lb, u, g.Bt * g.Hkv, g.B) - g.R;
+}
+__device__ __forceinline__ int32_t* unit_out(const SelGeom& g, int32_t* idx, int64_t u) {
+  return idx + unit_out_row(g.lb, u, g.Bt * g.Hkv, g.B);
 }
 
 // Average pooling: p_j = (1/k) * sum_{|t| <= k/2, 0 <= j+t < Ls} c_{j+t} (zero padding, divisor
@@ -162,7 +170,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
                                                              int32_t* __restrict__ idx,
                                                              const __grid_constant__ SelGeom g) {
   const int64_t u = blockIdx.x;
-  select_unit(pooled + u * (int64_t)g.Ls_full, idx + u * (int64_t)g.B, unit_scored(g, u), g.Kb, g.R);
+  select_unit(pooled + u * (int64_t)g.Ls_full, unit_out(g, idx, u), unit_scored(g, u), unit_kb(g, u), g.R);
 }
 
 // Steps 4 and 5 in one pass over the column sums: the block pools its unit's scores into shared
@@ -184,7 +192,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const float* _
     if (pooled_out) pooled_out[u * (int64_t)g.Ls_full + j] = pj;
   }
   __syncthreads();
-  select_unit(s_pooled, idx + u * (int64_t)g.B, Ls, g.Kb, g.R);
+  select_unit(s_pooled, unit_out(g, idx, u), Ls, unit_kb(g, u), g.R);
 }
 
 // Steps 4 and 5 for units of at most kRegItems * 1024 scored positions, with the unit's pooled
@@ -229,8 +237,8 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads) pool_select_reg_ker
   __shared__ uint32_t s_gt[kWarps], s_eq[kWarps];
   extern __shared__ __align__(16) float s_c[];  // the unit's column sums, [0, Ls) rounded up to 4
   const int64_t u = blockIdx.x;
-  const int Ls = unit_scored(g, u), Kb = g.Kb, R = g.R;
-  int32_t* out = idx + u * (int64_t)g.B;
+  const int Ls = unit_scored(g, u), Kb = unit_kb(g, u), R = g.R;
+  int32_t* out = unit_out(g, idx, u);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // One coalesced pass brings the column sums on chip (rows are 512-byte aligned and padded to
   // a multiple of 128 floats); the pooling taps then read shared memory instead of L1/L2.
@@ -336,8 +344,9 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads) pool_select_reg_ker
 
 static SelGeom sel_geom(const Dims& d) {
   SelGeom g;
-  g.Ls_full = d.Ls; g.Kb = d.Kb; g.R = d.R; g.B = d.B; g.Bt = d.Bt; g.Hkv = d.Hkv;
+  g.Ls_full = d.Ls; g.R = d.R; g.B = d.B; g.Bt = d.Bt; g.Hkv = d.Hkv;
   g.sl = d.sl;
+  g.lb = d.lb;
   return g;
 }
 

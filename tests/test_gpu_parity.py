@@ -476,11 +476,11 @@ def test_recall_of_two_selections_matches_oracle(laq):
 
 
 def test_layer_wise_budgets_on_layer_slices(laq):
-    # a pyramid of budgets: each run of equal budgets is one call on a slice of the layer dimension
+    # a pyramid of budgets, read back through the per-layer views of the ragged pool
     NL, Bt, Hq, Hkv, D, L, W, kernel = 4, 1, 4, 2, 128, 640, 8, 7
     budgets = [96, 96, 48, 24]
     q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=61)
-    outs = laq.evict_layer_budgets(q.cuda(), k.cuda(), v.cuda(), budgets, pool_kernel=kernel)
+    outs = laq.evict_layer_budgets(q.cuda(), k.cuda(), v.cuda(), budgets, pool_kernel=kernel)["layers"]
     torch.cuda.synchronize()
     for n, B in enumerate(budgets):
         ref = orc.evict(q[n:n + 1], k[n:n + 1], v[n:n + 1], W, kernel, B)
@@ -534,6 +534,66 @@ def test_workspace_reuse_back_to_back(laq):
 
 
 # ---------------------------------------------------------------- the paper-shaped configs
+def test_per_layer_budgets_write_one_ragged_pool(laq):
+    # a pyramid of budgets; with and without per-prompt lengths; every layer against the oracle
+    NL, Bt, Hq, Hkv, D, L, W, kernel = 4, 2, 8, 2, 128, 1100, 8, 7
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=71, kscale=1.5)
+    for budgets, lens in (([160, 128, 96, 64], None), ([64, 300, 64, 65], [1100, 700])):
+        out = laq.evict_layer_budgets(q.cuda(), k.cuda(), v.cuda(), budgets, pool_kernel=kernel,
+                                      seq_lens=lens)
+        assert laq.laq_last_device_status(out["params"], out["ws"]) == laq.LAQ_OK
+        ref = orc.evict_layers(q, k, v, W, kernel, budgets, seq_lens=lens)
+        got_idx = out["idx"].cpu().numpy()
+        assert got_idx.shape == ref["idx"].shape
+        kb, vb = bits(k), bits(v)
+        ko, vo = bits(out["k_out"]), bits(out["v_out"])
+        row = 0
+        for n, B in enumerate(budgets):
+            for b in range(Bt):
+                Lb = L if lens is None else lens[b]
+                for h in range(Hkv):
+                    gi = got_idx[row:row + B]
+                    check_index_set(gi, ref["idx"][row:row + B], ref["scores"][n, b, h][:Lb - W], Lb, W, B)
+                    assert (ko[row:row + B] == kb[n, b, h][gi]).all()
+                    assert (vo[row:row + B] == vb[n, b, h][gi]).all()
+                    row += B
+        assert row == got_idx.shape[0]
+    # equal budgets give exactly what laq_evict gives
+    uni = run_evict(laq, q, k, v, W, kernel, 100)
+    same = laq.evict_layer_budgets(q.cuda(), k.cuda(), v.cuda(), [100] * NL, pool_kernel=kernel)
+    assert torch.equal(same["idx"].view_as(uni["idx"]), uni["idx"])
+    assert torch.equal(same["k_out"].view_as(uni["k_out"]), uni["k_out"])
+    # host-side validation: the largest budget must be the one that sized the workspace
+    p = laq.params_for(q.cuda(), k.cuda(), W, kernel, 100, v=v.cuda())
+    assert laq.laq_layers_pool_entries(p, [100, 50, 120, 60]) == 0
+    assert laq.laq_layers_pool_entries(p, [100, 50, W, 60]) == 0
+
+
+def test_streaming_keep_set_and_its_compaction(laq):
+    NL, Bt, Hq, Hkv, D, L, W, B, n_sink = 2, 3, 4, 2, 128, 500, 4, 48, 4
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=72)
+    kd, vd = k.cuda(), v.cuda()
+    for lens in (None, [500, 333, 49]):
+        p = laq.params_for(q.cuda(), kd, W, 7, B, v=vd)
+        p.set_seq_lens(lens)
+        idx = torch.empty((NL, Bt, Hkv, B), dtype=torch.int32, device="cuda")
+        laq.laq_streaming_indices(p, n_sink, idx)
+        k_out = torch.empty((NL, Bt, Hkv, B, D), dtype=torch.bfloat16, device="cuda")
+        v_out = torch.empty_like(k_out)
+        laq.laq_compact(p, kd, vd, idx, k_out, v_out)
+        got = idx.cpu().numpy()
+        for b in range(Bt):
+            want = orc.streaming_indices(L, B, n_sink, None if lens is None else lens[b])
+            for n in range(NL):
+                for h in range(Hkv):
+                    assert (got[n, b, h] == want).all()
+                    assert (bits(k_out[n, b, h]) == orc.compact(k[n, b, h], want)).all()
+                    assert (bits(v_out[n, b, h]) == orc.compact(v[n, b, h], want)).all()
+    p = laq.params_for(q.cuda(), kd, W, 7, B, v=vd)
+    assert laq.laq_streaming_indices(p, B + 1, idx, check=False) == laq.LAQ_ERR_INVALID_ARG
+    assert laq.laq_streaming_indices(p, -1, idx, check=False) == laq.LAQ_ERR_INVALID_ARG
+
+
 def test_config1_full_with_planted_key(laq):
     cfg = synth.CONFIGS[1]
     inp = synth.make_inputs(cfg, "cpu")

@@ -495,3 +495,56 @@ def test_seq_lens_equal_separate_runs_on_truncated_prompts():
         assert (out["idx"][:, b, :, B - R:] == np.arange(Lb - R, Lb)).all()
         assert (out["k_out"][:, b] == ref["k_out"][:, 0]).all()
         assert (out["v_out"][:, b] == ref["v_out"][:, 0]).all()
+
+
+# ---------------------------------------------------------------- per-layer budgets, streaming keep-set
+def test_layer_budgets_identical_keys_closed_form_and_pool_layout():
+    # identical keys in every layer: layer n keeps [k/2, k/2 + B_n - R) and the tail, whatever its
+    # queries are; the ragged pool holds the layers end to end, [Bt][Hkv][B_n] entries each
+    NL, Bt, Hq, Hkv, W, D, L, R, kernel = 3, 2, 4, 2, 4, 16, 64, 4, 7
+    budgets = [20, 9, 33]
+    q = rand_bf16((NL, Bt, Hq, W, D), 61)
+    k = bf16(torch.ones((NL, Bt, Hkv, L, D)) * 0.25)
+    v = rand_bf16((NL, Bt, Hkv, L, D), 62)
+    out = orc.evict_layers(q, k, v, R, kernel, budgets)
+    assert out["idx"].shape == (Bt * Hkv * sum(budgets),)
+    row = 0
+    vb = v.view(torch.int16).numpy().view(np.uint16)
+    for n, B in enumerate(budgets):
+        want = list(range(kernel // 2, kernel // 2 + (B - R))) + list(range(L - R, L))
+        for b in range(Bt):
+            for h in range(Hkv):
+                got = out["idx"][row:row + B]
+                assert got.tolist() == want, (n, b, h)
+                assert (out["v_out"][row:row + B] == vb[n, b, h][got]).all()
+                row += B
+    assert row == out["idx"].shape[0]
+
+
+def test_layer_budgets_nest_when_layers_hold_the_same_cache():
+    # the same queries and keys in every layer: a smaller budget keeps a subset of a larger one,
+    # and each layer equals a uniform run with its own budget
+    NL, W, D, L, R, kernel = 3, 4, 32, 200, 4, 5
+    q1, k1 = rand_bf16((1, 1, 2, W, D), 63), rand_bf16((1, 1, 1, L, D), 64, 1.5)
+    q, k = q1.repeat(NL, 1, 1, 1, 1), k1.repeat(NL, 1, 1, 1, 1)
+    budgets = [12, 40, 25]
+    out = orc.evict_layers(q, k, None, R, kernel, budgets, fast_select=False)
+    sets, row = [], 0
+    for B in budgets:
+        sets.append(set(out["idx"][row:row + B].tolist()))
+        assert len(sets[-1]) == B
+        row += B
+    assert sets[0] < sets[2] < sets[1]
+    uni = orc.evict(q1, k1, None, R, kernel, 25, fast_select=False)
+    assert sets[2] == set(uni["idx"][0, 0, 0].tolist())
+
+
+def test_streaming_keep_set_structure():
+    for L, B, ns, Lb in [(100, 10, 4, None), (100, 10, 0, None), (100, 10, 10, None), (100, 30, 4, 57)]:
+        idx = orc.streaming_indices(L, B, ns, Lb)
+        end = L if Lb is None else Lb
+        assert idx.shape == (B,) and (np.diff(idx) > 0).all()
+        assert idx[:ns].tolist() == list(range(ns))
+        if ns < B:
+            assert idx[-1] == end - 1 and idx[ns] == end - (B - ns)
+        assert set(idx.tolist()) == set(range(ns)) | set(range(end - (B - ns), end))
