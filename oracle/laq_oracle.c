@@ -92,6 +92,38 @@ void laq_oracle_unit_colsum_local(const uint16_t* q, const uint16_t* k, int G, i
 }
 
 /*
+ * Column sums of each query head on its own: c_heads[g][j] = sum_{i<W} P[(g,i)][j]. The rows of
+ * different heads do not interact (every row has its own softmax), so head g is the unit
+ * computation above with that head's W queries alone. Row g of c_heads starts at g*row_stride.
+ */
+void laq_oracle_unit_colsum_heads(const uint16_t* q, const uint16_t* k, int G, int W, int W_local,
+                                  int D, int L, double scale, double* c_heads, int64_t row_stride) {
+  for (int g = 0; g < G; ++g)
+    laq_oracle_unit_colsum_local(q + (size_t)g * W * D, k, 1, W, W_local, D, L, scale,
+                                 c_heads + g * row_stride, NULL, NULL);
+}
+
+/*
+ * How the G query heads that share a KV head are combined into one importance per key (the
+ * paper does not define it): mode 0 adds them (the reading used throughout), mode 1 takes the
+ * largest, so that a key one head attends to strongly is not averaged away by the others.
+ */
+void laq_oracle_group_reduce(const double* c_heads, int G, int L, int mode, double* c) {
+  for (int j = 0; j < L; ++j) {
+    double acc = c_heads[j];
+    for (int g = 1; g < G; ++g) {
+      const double x = c_heads[(size_t)g * L + j];
+      if (mode == 1) {
+        if (x > acc) acc = x;
+      } else {
+        acc += x;
+      }
+    }
+    c[j] = acc;
+  }
+}
+
+/*
  * Step 4: average pooling over the scored positions [0, Ls), stride 1, zero padding of k/2 on
  * both sides, divisor always k (SnapKV-style pooling, Section 5.1 "employs average pooling").
  */
@@ -222,13 +254,17 @@ void laq_oracle_compact(const uint16_t* src, const int32_t* idx, int B, int D, u
  *   W_local    unified window of LAQ++ (Eq. 5), see laq_oracle_unit_colsum_local
  *   pool_mode  0 average pooling, 1 maximum pooling
  *   score_mode 0 attention weights (softmax), 1 raw logit sums (Eq. 4 read literally)
+ *   group_mode 0: the G heads of a group are summed (one kept set per KV head); 1: the largest
+ *              head counts (one kept set per KV head); 2: every query head selects for itself:
+ *              scores are then [NL][Bt][Hq][L-R], idx [NL][Bt][Hq][B], k_out / v_out
+ *              [NL][Bt][Hq][B][D], head h*G+g gathering from KV head h (softmax scoring only)
  *   seq_lens   [Bt] or NULL: prompt b holds only its first seq_lens[b] <= L positions. Everything
  *              is then taken relative to that length Lb: keys [0, Lb), local queries at the last
  *              W_local of them, scored positions [0, Lb-R), tail [Lb-R, Lb). Scores and column
  *              sums beyond are written as 0; rows of K/V beyond Lb are never read.
  */
 typedef struct {
-  int32_t W_local, pool_mode, score_mode, reserved;
+  int32_t W_local, pool_mode, score_mode, group_mode;
   const int32_t* seq_lens;
 } laq_oracle_variant;
 
@@ -278,7 +314,38 @@ int laq_oracle_evict_variant(const uint16_t* q, const uint16_t* k, const uint16_
     const int Ls = Lb - R;
     double* c = (double*)calloc((size_t)L, sizeof(double));
     double* p = (double*)calloc((size_t)(L - R > 0 ? L - R : 1), sizeof(double));
-    if (var->score_mode == 1)
+    if (var->group_mode != 0 && var->score_mode == 0) {
+      /* per-head column sums, then either their maximum or one selection per query head */
+      double* ch = (double*)calloc((size_t)G * L, sizeof(double));
+      laq_oracle_unit_colsum_heads(qu, ku, G, W, var->W_local, D, Lb, scale, ch, L);
+      if (var->group_mode == 2) {
+        for (int g = 0; g < G; ++g) {
+          const int64_t uh = u * G + g; /* (layer*Bt + b)*Hq + h*G + g */
+          const double* cg = ch + (size_t)g * L;
+          if (var->pool_mode == 1)
+            laq_oracle_pool_max(cg, Ls, kernel, p);
+          else
+            laq_oracle_pool(cg, Ls, kernel, p);
+          if (colsum) memcpy(colsum + uh * (int64_t)L, cg, (size_t)L * sizeof(double));
+          if (scores) memcpy(scores + uh * (int64_t)(L - R), p, (size_t)(L - R) * sizeof(double));
+          if (idx) {
+            int32_t* iu = idx + uh * (int64_t)B;
+            if (fast_select)
+              laq_oracle_select_sorted(p, Lb, R, B, iu);
+            else
+              laq_oracle_select(p, Lb, R, B, iu);
+            if (k_out) laq_oracle_compact(ku, iu, B, D, k_out + uh * (int64_t)B * D);
+            if (v_out) laq_oracle_compact(v + u * (int64_t)L * D, iu, B, D, v_out + uh * (int64_t)B * D);
+          }
+        }
+        free(ch);
+        free(c);
+        free(p);
+        continue;
+      }
+      laq_oracle_group_reduce(ch, G, L, var->group_mode, c);
+      free(ch);
+    } else if (var->score_mode == 1)
       laq_oracle_unit_rawsum(qu, ku, G, W, D, Lb, scale, c);
     else
       laq_oracle_unit_colsum_local(qu, ku, G, W, var->W_local, D, Lb, scale, c, NULL, NULL);

@@ -28,7 +28,7 @@ def build(force: bool = False) -> str:
 
 class _Variant(ctypes.Structure):
     _fields_ = [("W_local", ctypes.c_int32), ("pool_mode", ctypes.c_int32),
-                ("score_mode", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("score_mode", ctypes.c_int32), ("group_mode", ctypes.c_int32),
                 ("seq_lens", ctypes.c_void_p)]
 
 
@@ -65,6 +65,10 @@ def _load():
                                                  ctypes.POINTER(_Variant), vp, i64,
                                                  vp, vp, vp, vp, vp, i]
         lib.laq_oracle_evict_variant.restype = i
+        lib.laq_oracle_unit_colsum_heads.argtypes = [vp, vp, i, i, i, i, i, d, vp, i64]
+        lib.laq_oracle_unit_colsum_heads.restype = None
+        lib.laq_oracle_group_reduce.argtypes = [vp, i, i, i, vp]
+        lib.laq_oracle_group_reduce.restype = None
         _lib = lib
     return _lib
 
@@ -100,6 +104,26 @@ def unit_colsum(q, k, scale=None, local_window=0):
     _load().laq_oracle_unit_colsum_local(_ptr(q), _ptr(k), G, W, int(local_window), D, L, scale,
                                          _ptr(c), _ptr(m), _ptr(l))
     return c, m, l
+
+
+def unit_colsum_heads(q, k, scale=None, local_window=0):
+    """q [G][W][D], k [L][D] bf16 -> c_heads [G][L]: the column sums of every query head on its own."""
+    q, k = _bits(q), _bits(k)
+    G, W, D = q.shape
+    L = k.shape[0]
+    scale = 1.0 / np.sqrt(D) if scale is None else float(scale)
+    ch = np.zeros((G, L), np.float64)
+    _load().laq_oracle_unit_colsum_heads(_ptr(q), _ptr(k), G, W, int(local_window), D, L, scale,
+                                         _ptr(ch), L)
+    return ch
+
+
+def group_reduce(c_heads, mode):
+    """[G][L] per-head column sums -> [L]: mode 0 adds the heads, mode 1 takes the largest."""
+    ch = np.ascontiguousarray(c_heads, np.float64)
+    c = np.empty(ch.shape[1], np.float64)
+    _load().laq_oracle_group_reduce(_ptr(ch), ch.shape[0], ch.shape[1], int(mode), _ptr(c))
+    return c
 
 
 def pool(c, Ls, kernel, mode=0):
@@ -151,14 +175,16 @@ def compact(src, idx):
 
 
 def evict(q, k, v, R, kernel, B, scale=None, units=None, want_colsum=False, fast_select=True,
-          want_idx=True, local_window=0, pool_mode=0, score_mode=0, seq_lens=None):
+          want_idx=True, local_window=0, pool_mode=0, score_mode=0, seq_lens=None, group_mode=0):
     """Whole step on dense tensors. q [NL][Bt][Hq][W][D], k/v [NL][Bt][Hkv][L][D] (bf16).
 
     Returns a dict with 'scores' [NL,Bt,Hkv,L-R] fp64, 'idx' [NL,Bt,Hkv,B] int32, 'k_out',
     'v_out' [NL,Bt,Hkv,B,D] uint16 bit patterns, 'threads', and 'colsum' if asked. With `units`
     (unit numbers (layer*Bt+b)*Hkv+h) only those units are computed; the rest stays zero.
     `pool_mode` 1 pools by maximum, `score_mode` 1 sums raw logits instead of attention weights,
-    `seq_lens` [Bt] gives every prompt its own length (<= L).
+    `seq_lens` [Bt] gives every prompt its own length (<= L). `group_mode` 1 combines the query
+    heads of a group by maximum instead of sum; 2 lets every query head select for itself, and the
+    outputs then have Hq in place of Hkv.
     """
     q, k = _bits(q), _bits(k)
     v = None if v is None else _bits(v)
@@ -167,15 +193,17 @@ def evict(q, k, v, R, kernel, B, scale=None, units=None, want_colsum=False, fast
     assert k.shape == (NL, Bt, Hkv, L, D) and Hq % Hkv == 0
     scale = 1.0 / np.sqrt(D) if scale is None else float(scale)
     Ls = L - R
-    scores = np.zeros((NL, Bt, Hkv, Ls), np.float64)
-    colsum = np.zeros((NL, Bt, Hkv, L), np.float64) if want_colsum else None
-    idx = np.zeros((NL, Bt, Hkv, B), np.int32) if want_idx else None
-    k_out = np.zeros((NL, Bt, Hkv, B, D), np.uint16) if want_idx else None
-    v_out = np.zeros((NL, Bt, Hkv, B, D), np.uint16) if (want_idx and v is not None) else None
+    Ho = Hq if group_mode == 2 else Hkv   # heads of the outputs
+    scores = np.zeros((NL, Bt, Ho, Ls), np.float64)
+    colsum = np.zeros((NL, Bt, Ho, L), np.float64) if want_colsum else None
+    idx = np.zeros((NL, Bt, Ho, B), np.int32) if want_idx else None
+    k_out = np.zeros((NL, Bt, Ho, B, D), np.uint16) if want_idx else None
+    v_out = np.zeros((NL, Bt, Ho, B, D), np.uint16) if (want_idx and v is not None) else None
     ul = None if units is None else np.ascontiguousarray(units, np.int64)
     sl = None if seq_lens is None else np.ascontiguousarray(seq_lens, np.int32)
     assert sl is None or (sl.shape == (Bt,) and (sl <= L).all() and (sl > B).all())
-    var = _Variant(int(local_window), int(pool_mode), int(score_mode), 0, _ptr(sl))
+    assert group_mode == 0 or score_mode == 0
+    var = _Variant(int(local_window), int(pool_mode), int(score_mode), int(group_mode), _ptr(sl))
     threads = _load().laq_oracle_evict_variant(
         _ptr(q), _ptr(k), _ptr(v), NL, Bt, Hq, Hkv, D, L, W, R, kernel, B, scale, ctypes.byref(var),
         _ptr(ul), 0 if ul is None else ul.shape[0], _ptr(scores), _ptr(colsum), _ptr(idx), _ptr(k_out),

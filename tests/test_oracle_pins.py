@@ -548,3 +548,60 @@ def test_streaming_keep_set_structure():
         if ns < B:
             assert idx[-1] == end - 1 and idx[ns] == end - (B - ns)
         assert set(idx.tolist()) == set(range(ns)) | set(range(end - (B - ns), end))
+
+
+# ---------------------------------------------------------------- how the heads of a GQA group combine
+def test_per_head_column_sums_against_library_softmax_and_the_group_sum():
+    G, W, D, L = 4, 3, 32, 150
+    q, k = rand_bf16((G, W, D), 81), rand_bf16((L, D), 82, 1.5)
+    ch = orc.unit_colsum_heads(q, k)
+    assert ch.shape == (G, L)
+    s = (q.double().reshape(G, W, D) @ k.double().T) / math.sqrt(D)   # [G, W, L]
+    want = torch.softmax(s, dim=-1).sum(1).numpy()
+    np.testing.assert_allclose(ch, want, rtol=1e-12)
+    np.testing.assert_allclose(ch.sum(1), W, rtol=1e-12)           # W probability rows per head
+    c_all, _, _ = orc.unit_colsum(q, k)                               # the G-head statement
+    np.testing.assert_allclose(orc.group_reduce(ch, 0), c_all, rtol=1e-12)
+    np.testing.assert_allclose(orc.group_reduce(ch, 1), want.max(0), rtol=1e-12)
+    # max <= sum <= G * max, and one head alone is both
+    mx, sm = orc.group_reduce(ch, 1), orc.group_reduce(ch, 0)
+    assert (mx <= sm).all() and (sm <= G * mx * (1 + 1e-12)).all()
+    one = orc.unit_colsum_heads(q[:1], k)
+    np.testing.assert_array_equal(orc.group_reduce(one, 1), orc.group_reduce(one, 0))
+
+
+def test_group_max_mode_selects_on_the_largest_head():
+    NL, Bt, Hq, Hkv, W, D, L, R, kernel, B = 1, 2, 6, 2, 4, 32, 120, 4, 5, 30
+    q, k, v = rand_bf16((NL, Bt, Hq, W, D), 83), rand_bf16((NL, Bt, Hkv, L, D), 84, 1.5), rand_bf16((NL, Bt, Hkv, L, D), 85)
+    out = orc.evict(q, k, v, R, kernel, B, group_mode=1, want_colsum=True, fast_select=False)
+    G = Hq // Hkv
+    for b in range(Bt):
+        for h in range(Hkv):
+            s = (q[0, b, h * G:(h + 1) * G].double() @ k[0, b, h].double().T) / math.sqrt(D)
+            c = torch.softmax(s, dim=-1).sum(1).max(0).values          # [L]
+            np.testing.assert_allclose(out["colsum"][0, b, h], c.numpy(), rtol=1e-12)
+            p = torch.nn.functional.avg_pool1d(c[None, None, :L - R], kernel, 1, kernel // 2,
+                                               count_include_pad=True)[0, 0]
+            np.testing.assert_allclose(out["scores"][0, b, h], p.numpy(), rtol=1e-12)
+            order = np.argsort(-out["scores"][0, b, h], kind="stable")[:B - R]
+            assert out["idx"][0, b, h].tolist() == sorted(order.tolist()) + list(range(L - R, L))
+
+
+def test_per_query_head_selection_is_the_step_with_every_head_as_its_own_group():
+    # replicate each KV head for its G query heads: the per-head mode on the GQA problem must give
+    # what the plain step gives on that expanded problem
+    NL, Bt, Hq, Hkv, W, D, L, R, kernel, B = 2, 1, 4, 2, 3, 16, 90, 3, 3, 25
+    G = Hq // Hkv
+    q, k, v = rand_bf16((NL, Bt, Hq, W, D), 86), rand_bf16((NL, Bt, Hkv, L, D), 87, 2.0), rand_bf16((NL, Bt, Hkv, L, D), 88)
+    got = orc.evict(q, k, v, R, kernel, B, group_mode=2, fast_select=False)
+    k_rep, v_rep = k.repeat_interleave(G, dim=2), v.repeat_interleave(G, dim=2)
+    want = orc.evict(q, k_rep, v_rep, R, kernel, B, fast_select=False)
+    assert got["idx"].shape == (NL, Bt, Hq, B)
+    np.testing.assert_array_equal(got["idx"], want["idx"])
+    np.testing.assert_array_equal(got["scores"], want["scores"])
+    np.testing.assert_array_equal(got["k_out"], want["k_out"])
+    np.testing.assert_array_equal(got["v_out"], want["v_out"])
+    # with per-prompt lengths too
+    got = orc.evict(q, k, v, R, kernel, B, group_mode=2, seq_lens=[70])
+    want = orc.evict(q, k_rep, v_rep, R, kernel, B, seq_lens=[70])
+    np.testing.assert_array_equal(got["idx"], want["idx"])
