@@ -91,6 +91,15 @@ typedef enum { LAQ_POOL_AVG = 0, LAQ_POOL_MAX = 1 } laq_pool_mode;
  * negative; local_window has no effect because it only masks positions inside the tail). */
 typedef enum { LAQ_SCORE_SOFTMAX = 0, LAQ_SCORE_RAW = 1 } laq_score_mode;
 
+/* How the G query heads that share a KV head are combined (the paper's Eq. 4 does not say; its
+ * models are GQA models). LAQ_GROUP_SUM: the column sums of the group's heads are added, one kept
+ * set per KV head (the reading used throughout). LAQ_GROUP_MAX: per key the largest head's column
+ * sum counts, one kept set per KV head. LAQ_GROUP_PER_HEAD: every query head ranks and keeps for
+ * itself; scores, idx, K_out and V_out then have Hq in place of Hkv in their shapes (query head
+ * h*G+g gathers from KV head h; the o_stride_head stride steps over query heads). The last two
+ * need LAQ_SCORE_SOFTMAX. */
+typedef enum { LAQ_GROUP_SUM = 0, LAQ_GROUP_MAX = 1, LAQ_GROUP_PER_HEAD = 2 } laq_group_mode;
+
 /* Problem description. Plain data; copy freely. All strides are in bf16 ELEMENTS. */
 typedef struct {
   int32_t n_layers;    /* NL >= 1 */
@@ -116,6 +125,8 @@ typedef struct {
    * local_window <= keep_tail, so that every scored position is visible to every query. */
   int32_t local_window;
   int32_t score_mode;      /* laq_score_mode */
+  int32_t group_mode;      /* laq_group_mode */
+  int32_t reserved0;       /* must be 0 */
   /* Q [NL][Bt][Hq][W][D] */
   int64_t q_stride_layer, q_stride_batch, q_stride_head, q_stride_pos;
   /* K [NL][Bt][Hkv][L][D] */

@@ -24,6 +24,7 @@ LAQ_ERR_TIMEOUT = 5
 LAQ_ERR_INTERNAL = 6
 LAQ_POOL_AVG, LAQ_POOL_MAX = 0, 1
 LAQ_SCORE_SOFTMAX, LAQ_SCORE_RAW = 0, 1
+LAQ_GROUP_SUM, LAQ_GROUP_MAX, LAQ_GROUP_PER_HEAD = 0, 1, 2
 
 EXPORTS = (
     "laq_params_dense_strides", "laq_workspace_bytes", "laq_score", "laq_select", "laq_compact",
@@ -41,7 +42,8 @@ class LaqParams(ctypes.Structure):
         "n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "prompt_len", "window_len",
         "keep_tail", "pool_kernel", "pool_mode", "budget")] + [("softmax_scale", ctypes.c_float),
         ("tiles_per_task", ctypes.c_int32), ("sched_lag_tasks", ctypes.c_int32),
-        ("local_window", ctypes.c_int32), ("score_mode", ctypes.c_int32)] + [
+        ("local_window", ctypes.c_int32), ("score_mode", ctypes.c_int32),
+        ("group_mode", ctypes.c_int32), ("reserved0", ctypes.c_int32)] + [
         (f"{t}_stride_{d}", ctypes.c_int64) for t in ("q", "k", "v", "o")
         for d in ("layer", "batch", "head", "pos")] + [("seq_lens", ctypes.POINTER(ctypes.c_int32))]
 
@@ -272,22 +274,26 @@ def laq_version() -> int:
 def evict(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, budget: int, pool_kernel: int = 7,
           keep_tail: Optional[int] = None, want_scores: bool = False, ws=None, stream=None,
           softmax_scale: float = 0.0, local_window: int = 0, pool_mode: int = 0,
-          score_mode: int = 0, seq_lens=None):
+          score_mode: int = 0, seq_lens=None, group_mode: int = 0):
     """Convenience call: allocates the outputs with torch and runs ``laq_evict``.
 
     q [NL,Bt,Hq,W,D], k and v [NL,Bt,Hkv,L,D], bf16 CUDA tensors. Returns a dict with 'k_out',
-    'v_out' [NL,Bt,Hkv,B,D], 'idx' [NL,Bt,Hkv,B] int32 and, if asked, 'scores' [NL,Bt,Hkv,L-R].
+    'v_out' [NL,Bt,Hkv,B,D], 'idx' [NL,Bt,Hkv,B] int32 and, if asked, 'scores' [NL,Bt,Hkv,L-R]
+    (with ``group_mode = LAQ_GROUP_PER_HEAD`` every query head selects for itself and the outputs
+    have Hq in place of Hkv).
     """
     if not (q.is_cuda and k.is_cuda and v.is_cuda):
         raise ValueError("evict: q, k and v must be CUDA tensors (there is no CPU path)")
     NL, Bt, Hq, W, D = q.shape
     Hkv, L = k.shape[2], k.shape[3]
     R = W if keep_tail is None else keep_tail
-    k_out = torch.empty((NL, Bt, Hkv, budget, D), dtype=k.dtype, device=k.device)
+    Ho = Hq if group_mode == LAQ_GROUP_PER_HEAD else Hkv
+    k_out = torch.empty((NL, Bt, Ho, budget, D), dtype=k.dtype, device=k.device)
     v_out = torch.empty_like(k_out)
-    idx = torch.empty((NL, Bt, Hkv, budget), dtype=torch.int32, device=k.device)
-    scores = torch.empty((NL, Bt, Hkv, L - R), dtype=torch.float32, device=k.device) if want_scores else None
+    idx = torch.empty((NL, Bt, Ho, budget), dtype=torch.int32, device=k.device)
+    scores = torch.empty((NL, Bt, Ho, L - R), dtype=torch.float32, device=k.device) if want_scores else None
     p = params_for(q, k, R, pool_kernel, budget, v=v, out=k_out)
+    p.group_mode = group_mode        # how the query heads of a GQA group combine
     p.softmax_scale = softmax_scale  # 0 selects 1/sqrt(head_dim)
     p.local_window = local_window    # > 0: LAQ++ unified window (Eq. 5)
     p.pool_mode = pool_mode          # LAQ_POOL_AVG / LAQ_POOL_MAX

@@ -17,6 +17,7 @@ struct CompactArgs {
   int64_t vs_layer, vs_batch, vs_head, vs_pos;
   int64_t os_layer, os_batch, os_head, os_pos;
   int Bt, Hkv, B, dv, L;
+  int kv_div;  // unit head h reads KV head h / kv_div (1 unless every query head is a unit)
   int64_t u0;  // first unit of this launch (units are launched in slabs of at most 65535)
   LayerBudgets lb;  // per-layer budgets: B is then the largest, and the outputs are one dense ragged pool
 };
@@ -39,8 +40,9 @@ __global__ void __launch_bounds__(256) compact_kernel(const __grid_constant__ Co
   if (blockIdx.x * kRowsPerBlock >= B) return;  // a layer with a smaller budget (block-uniform)
   const int64_t row = unit_out_row(a.lb, u, a.Bt * a.Hkv, a.B);
   const int32_t* idx = a.idx + row;
-  const uint4* kbase = a.k + layer * a.ks_layer + b * a.ks_batch + h * a.ks_head;
-  const uint4* vbase = a.v + layer * a.vs_layer + b * a.vs_batch + h * a.vs_head;
+  const int h_src = h / a.kv_div;
+  const uint4* kbase = a.k + layer * a.ks_layer + b * a.ks_batch + h_src * a.ks_head;
+  const uint4* vbase = a.v + layer * a.vs_layer + b * a.vs_batch + h_src * a.vs_head;
   const int64_t obase =
       a.lb.n > 0 ? row * a.dv : layer * a.os_layer + b * a.os_batch + h * a.os_head;
   const int64_t os_pos = a.lb.n > 0 ? a.dv : a.os_pos;
@@ -113,6 +115,7 @@ laq_status compact_launch(const laq_params& p, const Dims& d, const void* k, con
   a.os_head = p.o_stride_head / 8;   a.os_pos = p.o_stride_pos / 8;
   a.Bt = d.Bt; a.Hkv = d.Hkv; a.B = d.B; a.dv = d.D / 8; a.L = d.L;
   a.lb = d.lb;
+  a.kv_div = d.kv_div > 0 ? d.kv_div : 1;
   // units sit on grid.y, which holds at most 65535 blocks
   for (int64_t u0 = 0; u0 < d.U; u0 += 65535) {
     a.u0 = u0;

@@ -38,8 +38,10 @@ laq_status derive_dims(const laq_params* p, Dims* d) {
   if (p->local_window < 0 || p->local_window > p->window_len || p->local_window > p->keep_tail)
     return LAQ_ERR_INVALID_ARG;
   if ((p->pool_mode != LAQ_POOL_AVG && p->pool_mode != LAQ_POOL_MAX) ||
-      (p->score_mode != LAQ_SCORE_SOFTMAX && p->score_mode != LAQ_SCORE_RAW))
+      (p->score_mode != LAQ_SCORE_SOFTMAX && p->score_mode != LAQ_SCORE_RAW) ||
+      p->group_mode < LAQ_GROUP_SUM || p->group_mode > LAQ_GROUP_PER_HEAD || p->reserved0 != 0)
     return LAQ_ERR_INVALID_ARG;
+  if (p->group_mode != LAQ_GROUP_SUM && p->score_mode != LAQ_SCORE_SOFTMAX) return LAQ_ERR_UNSUPPORTED;
   if ((p->head_dim % 8) != 0 || p->head_dim > 256) return LAQ_ERR_UNSUPPORTED;
   const int64_t M = (int64_t)(p->n_q_heads / p->n_kv_heads) * p->window_len;
   if (M > 256) return LAQ_ERR_UNSUPPORTED;
@@ -54,6 +56,8 @@ laq_status derive_dims(const laq_params* p, Dims* d) {
   d->W_local = p->local_window;
   d->pool_max = p->pool_mode == LAQ_POOL_MAX;
   d->score_raw = p->score_mode == LAQ_SCORE_RAW;
+  d->group_mode = p->group_mode;
+  d->kv_div = 1;
   d->R = p->keep_tail;
   d->kpool = p->pool_kernel;
   d->B = p->budget;
@@ -117,12 +121,17 @@ void plan_workspace(const Dims& d, int tiles_per_task, Workspace* w) {
   off = align_up(off + (size_t)d.U * w->M_pad * sizeof(float), 256);
   w->off_qsum = off;
   if (d.score_raw) off = align_up(off + (size_t)d.U * d.D * sizeof(float), 256);
+  // per-head column sums for the group modes that need them; with LAQ_GROUP_PER_HEAD they are
+  // the scores' source and the per-unit array is not used
+  w->off_colsum_h = off;
+  if (d.group_mode != LAQ_GROUP_SUM) off = align_up(off + (size_t)d.U * d.G * w->L_pad * sizeof(float), 256);
   w->off_colsum = off;
-  off = align_up(off + (size_t)d.U * w->L_pad * sizeof(float), 256);
+  if (d.group_mode != LAQ_GROUP_PER_HEAD) off = align_up(off + (size_t)d.U * w->L_pad * sizeof(float), 256);
+  const size_t sel_units = (size_t)d.U * (d.group_mode == LAQ_GROUP_PER_HEAD ? d.G : 1);
   w->off_pooled = off;
-  off = align_up(off + (size_t)d.U * d.Ls * sizeof(float), 256);
+  off = align_up(off + sel_units * d.Ls * sizeof(float), 256);
   w->off_idx = off;
-  off = align_up(off + (size_t)d.U * d.B * sizeof(int32_t), 256);
+  off = align_up(off + sel_units * d.B * sizeof(int32_t), 256);
   w->total = off;
 }
 
@@ -147,6 +156,29 @@ laq_status run_scoring(const laq_params* p, const Dims& d, const Workspace& w,
                             : score_simt_launch(*p, d, w, q, k, ws, stream, launches);
   if (g_ev_end && cudaEventRecord(g_ev_end, stream) != cudaSuccess) return LAQ_ERR_CUDA;
   return st;
+}
+
+Dims per_head_dims(const Dims& d) {
+  Dims dh = d;
+  dh.Hkv = d.Hq;
+  dh.G = 1;
+  dh.kv_div = d.G;
+  dh.U = d.U * d.G;
+  return dh;
+}
+
+laq_status selection_source(const Dims& d, const Workspace& w, char* ws, cudaStream_t stream,
+                            int* launches, const float** colsum, Dims* dsel) {
+  *dsel = d;
+  *colsum = (const float*)(ws + w.off_colsum);
+  if (d.group_mode == LAQ_GROUP_MAX)
+    return group_max_launch(d, (const float*)(ws + w.off_colsum_h), w.L_pad,
+                            (float*)(ws + w.off_colsum), stream, launches);
+  if (d.group_mode == LAQ_GROUP_PER_HEAD) {
+    *dsel = per_head_dims(d);
+    *colsum = (const float*)(ws + w.off_colsum_h);
+  }
+  return LAQ_OK;
 }
 
 static laq_status check_ws(const Workspace& w, const void* ws, size_t ws_bytes) {
@@ -207,8 +239,10 @@ laq_status laq_score(const laq_params* p, const void* q, const void* k, float* s
   char* wsb = (char*)ws;
   int launches = 0;
   st = run_scoring(p, d, w, q, k, wsb, stream, &launches);
-  if (st == LAQ_OK)
-    st = pool_launch(d, (const float*)(wsb + w.off_colsum), w.L_pad, scores, stream, &launches);
+  const float* colsum = nullptr;
+  Dims ds;
+  if (st == LAQ_OK) st = selection_source(d, w, wsb, stream, &launches, &colsum, &ds);
+  if (st == LAQ_OK) st = pool_launch(ds, colsum, w.L_pad, scores, stream, &launches);
   g_last_launches = launches;
   return st;
 }
@@ -282,18 +316,20 @@ static laq_status evict_impl(const laq_params* p, const Dims& d, const void* q, 
   int launches = 0;
   st = run_scoring(p, d, w, q, k, wsb, stream, &launches);
   int32_t* idx_dev = idx ? idx : (int32_t*)(wsb + w.off_idx);
-  const float* colsum = (const float*)(wsb + w.off_colsum);
+  const float* colsum = nullptr;
+  Dims ds;  // the sizes steps 4-6 see (every query head a unit of its own in the per-head mode)
+  if (st == LAQ_OK) st = selection_source(d, w, wsb, stream, &launches, &colsum, &ds);
   bool fused = false;
   if (st == LAQ_OK && (idx || k_out || v_out))
-    st = pool_select_launch(d, colsum, w.L_pad, scores, idx_dev, stream, &launches, &fused);
+    st = pool_select_launch(ds, colsum, w.L_pad, scores, idx_dev, stream, &launches, &fused);
   if (st == LAQ_OK && !fused) {
     float* pooled = scores ? scores : (float*)(wsb + w.off_pooled);
-    st = pool_launch(d, colsum, w.L_pad, pooled, stream, &launches);
+    st = pool_launch(ds, colsum, w.L_pad, pooled, stream, &launches);
     if (st == LAQ_OK && (idx || k_out || v_out))
-      st = select_launch(d, pooled, idx_dev, stream, &launches);
+      st = select_launch(ds, pooled, idx_dev, stream, &launches);
   }
   if (st == LAQ_OK && (k_out || v_out))
-    st = compact_launch(*p, d, k, v, idx_dev, k_out, v_out, stream, &launches);
+    st = compact_launch(*p, ds, k, v, idx_dev, k_out, v_out, stream, &launches);
   g_last_launches = launches;
   return st;
 }
@@ -321,7 +357,7 @@ static laq_status derive_layer_budgets(const laq_params* p, const int32_t* layer
       if (B >= d->sl.len[b]) return LAQ_ERR_INVALID_ARG;
     d->lb.B[n] = B;
     d->lb.row0[n] = row;
-    row += (int64_t)d->Bt * d->Hkv * B;
+    row += (int64_t)d->Bt * (d->group_mode == LAQ_GROUP_PER_HEAD ? d->Hq : d->Hkv) * B;
     if (B > largest) largest = B;
   }
   if (largest != p->budget) return LAQ_ERR_INVALID_ARG;
@@ -332,7 +368,8 @@ static laq_status derive_layer_budgets(const laq_params* p, const int32_t* layer
 size_t laq_layers_pool_entries(const laq_params* p, const int32_t* layer_budgets) {
   Dims d;
   if (derive_dims(p, &d) != LAQ_OK || derive_layer_budgets(p, layer_budgets, &d) != LAQ_OK) return 0;
-  return (size_t)(d.lb.row0[d.NL - 1] + (int64_t)d.Bt * d.Hkv * d.lb.B[d.NL - 1]);
+  return (size_t)(d.lb.row0[d.NL - 1] +
+                  (int64_t)d.Bt * (d.group_mode == LAQ_GROUP_PER_HEAD ? d.Hq : d.Hkv) * d.lb.B[d.NL - 1]);
 }
 
 laq_status laq_evict_layers(const laq_params* p, const int32_t* layer_budgets, const void* q,
@@ -417,6 +454,7 @@ laq_status laq_evict_host(const laq_params* p, const void* q_host, const void* k
   laq_status st = derive_dims(p, &d);
   if (st != LAQ_OK) return st;
   if (!q_host || !k_host || !v_host || !k_out_host || !v_out_host) return LAQ_ERR_INVALID_ARG;
+  if (d.group_mode == LAQ_GROUP_PER_HEAD) return LAQ_ERR_UNSUPPORTED;  // outputs are sized per KV head here
   HostStaging h;
   plan_staging(d, &h);
   if (!staging || (reinterpret_cast<uintptr_t>(staging) & 255u) != 0 || staging_bytes < h.total)

@@ -44,6 +44,9 @@ struct Dims {
   int W_local;  // leading causal queries of each head's window (LAQ++), 0 for plain LAQ
   int pool_max;   // 1: maximum pooling, 0: average pooling
   int score_raw;  // 1: raw logit sums (Eq. 4 read literally), 0: softmax column sums
+  int group_mode; // laq_group_mode: how the G heads of a unit combine
+  int kv_div;     // query heads per KV head as seen by the gather: 1, or G when every query head
+                  // is a unit of its own (per_head_dims) and head h reads KV head h / G
   int M;        // G*W softmax rows per unit
   int Ls, Kb;   // scored positions, selected slots
   int64_t U;    // units
@@ -59,11 +62,13 @@ struct Dims {
 //   part     : float2 [U][n_part][M_pad]  partial (max, sum) in the log2 domain, one per task
 //   row_off  : float [U][M_pad]  b_r = log2e*scale*m_r + log2(l_r) (CUDA-core path only)
 //   qsum     : float [U][D]  sum of the unit's query rows (raw-logit mode only)
+//   colsum_h : float [U*G][L_pad]  per-head column sums (group modes other than the sum only)
 //   colsum   : float [U][L_pad]  c_j (step 3)
 //   pooled   : float [U][Ls]     p_j (step 4) when the caller gave no scores buffer
 //   idx      : int32 [U][B]      kept positions when the caller gave no idx buffer
 struct Workspace {
-  size_t off_hdr, off_cnt, off_part, off_rowoff, off_qsum, off_colsum, off_pooled, off_idx, total;
+  size_t off_hdr, off_cnt, off_part, off_rowoff, off_qsum, off_colsum_h, off_colsum, off_pooled,
+      off_idx, total;
   int n_part;  // partial-statistics slots per unit = scoring tasks per unit and sweep
   int M_pad;   // rows padded to a multiple of 32
   int L_pad;   // L padded to a multiple of 128
@@ -88,6 +93,10 @@ laq_status check_strides_qk(const laq_params* p);
 laq_status run_scoring(const laq_params* p, const Dims& d, const Workspace& w, const void* q,
                        const void* k, char* ws, cudaStream_t stream, int* launches);
 void set_last_launch_count(int n);
+// After run_scoring: the column sums steps 4-6 read and the sizes they see. For LAQ_GROUP_MAX this
+// enqueues the maximum over the heads; for LAQ_GROUP_PER_HEAD every query head becomes a unit.
+laq_status selection_source(const Dims& d, const Workspace& w, char* ws, cudaStream_t stream,
+                            int* launches, const float** colsum, Dims* dsel);
 
 // Scoring back ends: both fill colsum (fp32 [U][L_pad]) on `stream`.
 // Tensor-core path (tcgen05 + TMA), head_dim 128, M <= 256.
@@ -100,6 +109,12 @@ laq_status score_raw_launch(const laq_params& p, const Dims& d, const Workspace&
 laq_status score_simt_launch(const laq_params& p, const Dims& d, const Workspace& w,
                              const void* q, const void* k, char* ws, cudaStream_t stream,
                              int* launches);
+
+// Elementwise maximum over the G per-head column sums of every unit (LAQ_GROUP_MAX).
+laq_status group_max_launch(const Dims& d, const float* colsum_h, int L_pad, float* colsum,
+                            cudaStream_t stream, int* launches);
+// The sizes seen by steps 4-6 when every query head selects for itself: Hq "KV heads", U*G units.
+Dims per_head_dims(const Dims& d);
 
 // Pool (step 4) from colsum into `pooled`.
 laq_status pool_launch(const Dims& d, const float* colsum, int L_pad, float* pooled,

@@ -20,6 +20,7 @@ struct SimtArgs {
   int64_t qs_layer, qs_batch, qs_head, qs_pos;
   int64_t ks_layer, ks_batch, ks_head, ks_pos;
   int Bt, Hkv, G, W, W_local, D, L, M, M_pad, n_part, L_pad, keys_per_chunk;
+  int per_head;  // 1: one column sum per query head, colsum is [U*G][L_pad]
   float scale_log2;  // softmax scale * log2(e)
   float2* part;
   float* row_off;
@@ -161,10 +162,15 @@ __global__ void simt_colsum_kernel(SimtArgs a) {
       for (int c = 0; c < dv; ++c)
         acc = dot8(sq[rr * stride4 + c], sk[threadIdx.x * stride4 + c], acc);
       sum += exp2f(fmaf(acc, a.scale_log2, -s_off[rr]));
+      if (a.per_head && (r0 + rr + 1) % a.W == 0) {  // last row of a query head
+        const int j = j0 + threadIdx.x;
+        if (j < Lu) a.colsum[(u * a.G + (r0 + rr) / a.W) * a.L_pad + j] = sum;
+        sum = 0.f;
+      }
     }
   }
   const int j = j0 + threadIdx.x;
-  if (j < Lu) a.colsum[u * a.L_pad + j] = sum;
+  if (!a.per_head && j < Lu) a.colsum[u * a.L_pad + j] = sum;
 }
 
 }  // namespace
@@ -185,7 +191,8 @@ laq_status score_simt_launch(const laq_params& p, const Dims& d, const Workspace
   a.scale_log2 = d.scale * kLog2e;
   a.part = (float2*)(ws + w.off_part);
   a.row_off = (float*)(ws + w.off_rowoff);
-  a.colsum = (float*)(ws + w.off_colsum);
+  a.per_head = d.group_mode != LAQ_GROUP_SUM;
+  a.colsum = (float*)(ws + (a.per_head ? w.off_colsum_h : w.off_colsum));
   a.sl = d.sl;
   if (d.U > 0x7fffffff || w.L_pad / kColTile > 65535) return LAQ_ERR_UNSUPPORTED;
   const int dv = d.D / 8;

@@ -65,8 +65,10 @@ extern "C" laq_status laq_score_static(const laq_params* p, const void* q, const
   // of the scratch is written before it is read
   int launches = 0;
   st = run_scoring(p, d, w, q, k, ws, stream, &launches);
-  if (st == LAQ_OK)
-    st = pool_launch(d, (const float*)(ws + w.off_colsum), w.L_pad, scores, stream, &launches);
+  const float* colsum = nullptr;
+  Dims ds;
+  if (st == LAQ_OK) st = selection_source(d, w, ws, stream, &launches, &colsum, &ds);
+  if (st == LAQ_OK) st = pool_launch(ds, colsum, w.L_pad, scores, stream, &launches);
   set_last_launch_count(launches);
   return st;
 }

@@ -427,7 +427,10 @@ __device__ __forceinline__ void stats_cols64(uint32_t taddr, float c, float& m, 
 // kDup: M <= 64, sweep 1 holds every query row twice (on TMEM lanes r and 64 + r).
 // kWide: 128 < M <= 256, two row blocks per tile, so an accumulator buffer takes 256 TMEM columns
 // and there are two K stages / buffers instead of four.
-template <bool kDup, bool kWide>
+// kPerHead: sweep 2 keeps one column sum per query head (colsum is [U*G][L_pad]); the launcher
+// only picks it when a head's rows never straddle a group of four rows or a 32-row chunk unevenly
+// (W a multiple of 4 that divides 32, or 32 or 64).
+template <bool kDup, bool kWide, bool kPerHead>
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
                 const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ TcArgs a) {
@@ -651,9 +654,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       // The column sums of this task's keys start at zero: sweep 2 adds into them with two
       // red.global per key. Zeroed here, before the fence and the counter bump below, they are
       // visible to every sweep-2 task of the unit, which waits for that counter.
-      {
-        float4* cz = reinterpret_cast<float4*>(a.colsum + (int64_t)task.unit * a.L_pad +
-                                               (int64_t)task.tile0 * TILE_KEYS);
+      for (int g = 0; g < (kPerHead ? a.G : 1); ++g) {
+        const int64_t row = kPerHead ? (int64_t)task.unit * a.G + g : (int64_t)task.unit;
+        float4* cz = reinterpret_cast<float4*>(a.colsum + row * a.L_pad + (int64_t)task.tile0 * TILE_KEYS);
         const int n4 = task.n_tiles * (TILE_KEYS / 4);
         for (int i = lane; i < n4; i += 32) cz[i] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
@@ -841,6 +844,30 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
             }
             release_buffer(empty_bar, lane);
           }
+        } else if (kPerHead) {
+          // one column sum per query head: the chunk's 32 rows come as eight groups of four, a
+          // head ends after every `gph` groups (all eight when a head spans whole chunks)
+          const int gph = (a.W < 32 ? a.W : 32) >> 2;
+          const int key = key0 + row_in_wg;
+#pragma unroll 1
+          for (int ch = ch_lo; ch < ch_hi; ++ch) {
+            tmem_ld32(taddr + (uint32_t)ch * 32u, v);
+            tmem_ld_wait(v);
+            if (ch + 1 == ch_hi) release_buffer(empty_bar, lane);
+            float hs[8];
+            colsum_groups(v, c, nboff + ch * 32, hs);
+            float run = 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              run += hs[i];
+              if (((i + 1) & (gph - 1)) == 0) {
+                const int g = (ch * 32 + 4 * i) / a.W;
+                if (key < Lu && g < a.G) red_add(&a.colsum[(u * a.G + g) * a.L_pad + key], run);
+                run = 0.f;
+              }
+            }
+          }
+          if (ch_lo == ch_hi) release_buffer(empty_bar, lane);
         } else {
           float2 acc[4];
 #pragma unroll
@@ -952,6 +979,11 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   // every chunk must hold at least one tile
   if ((a.tasks_per_unit - 1) * a.tiles_per_task >= a.n_tiles || d.W > 256 || d.G > 256)
     return score_simt_launch(p, d, w, q, k, ws, stream, launches);
+  // per-head column sums need every head's rows to fill whole groups of four inside the 32-row
+  // chunks, and at most two adds per (head, key) so that the result does not depend on their order
+  if (d.group_mode != LAQ_GROUP_SUM &&
+      !((d.W % 4 == 0 && 32 % d.W == 0) || d.W == 32 || d.W == 64))
+    return score_simt_launch(p, d, w, q, k, ws, stream, launches);
   if (d.U >= 0x7fffffff) return LAQ_ERR_UNSUPPORTED;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -994,7 +1026,7 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   a.hdr = (int32_t*)(ws + w.off_hdr);
   a.cnt = (int32_t*)(ws + w.off_cnt);
   a.part = (float2*)(ws + w.off_part);
-  a.colsum = (float*)(ws + w.off_colsum);
+  a.colsum = (float*)(ws + (d.group_mode != LAQ_GROUP_SUM ? w.off_colsum_h : w.off_colsum));
   a.sl = d.sl;
   const bool wide = d.M > 128;
   const int q_rows = wide ? 256 : 128, n_slots = wide ? 2 : 4;
@@ -1011,11 +1043,16 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
     return score_simt_launch(p, d, w, q, k, ws, stream, launches);  // layout TMA cannot describe
 
   const size_t smem = kCtlBytes + 2u * (size_t)q_rows * 256u + (size_t)n_slots * kKStageBytes;
-  auto kernel = dup ? score_tc_kernel<true, false>
-                    : (wide ? score_tc_kernel<false, true> : score_tc_kernel<false, false>);
+  const bool per_head = d.group_mode != LAQ_GROUP_SUM;
+  auto kernel = per_head ? (dup ? score_tc_kernel<true, false, true>
+                                : (wide ? score_tc_kernel<false, true, true>
+                                        : score_tc_kernel<false, false, true>))
+                         : (dup ? score_tc_kernel<true, false, false>
+                                : (wide ? score_tc_kernel<false, true, false>
+                                        : score_tc_kernel<false, false, false>));
   // the shared-memory opt-in is a per-device attribute of each kernel variant: set once
   static std::atomic<uint32_t> smem_opted_in[kMaxDevices];
-  const uint32_t variant_bit = 1u << (dup ? 0 : (wide ? 1 : 2));
+  const uint32_t variant_bit = 1u << ((dup ? 0 : (wide ? 1 : 2)) + (per_head ? 3 : 0));
   if (dev >= kMaxDevices || !(smem_opted_in[dev].load(std::memory_order_acquire) & variant_bit)) {
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)

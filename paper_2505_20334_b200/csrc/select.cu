@@ -340,7 +340,36 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads) pool_select_reg_ker
   for (int t = tid; t < R; t += kThreads) out[Kb + t] = Ls + t;
 }
 
+// c[u][j] = max over the G heads of c_h[u*G + g][j] (LAQ_GROUP_MAX); rows are L_pad floats,
+// a multiple of 128, read and written four at a time.
+__global__ void group_max_kernel(const float4* __restrict__ colsum_h, float4* __restrict__ colsum,
+                                 int row4, int G, int64_t total4) {
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= total4) return;
+  const int64_t u = i / row4;
+  const int j = (int)(i % row4);
+  const float4* src = colsum_h + u * G * (int64_t)row4 + j;
+  float4 m = __ldcs(src);
+  for (int g = 1; g < G; ++g) {
+    const float4 x = __ldcs(src + g * (int64_t)row4);
+    m.x = fmaxf(m.x, x.x); m.y = fmaxf(m.y, x.y); m.z = fmaxf(m.z, x.z); m.w = fmaxf(m.w, x.w);
+  }
+  colsum[i] = m;
+}
+
 }  // namespace
+
+laq_status group_max_launch(const Dims& d, const float* colsum_h, int L_pad, float* colsum,
+                            cudaStream_t stream, int* launches) {
+  const int row4 = L_pad / 4;
+  const int64_t total4 = d.U * (int64_t)row4;
+  const int64_t blocks = (total4 + 255) / 256;
+  if (blocks > 0x7fffffff) return LAQ_ERR_UNSUPPORTED;
+  group_max_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const float4*)colsum_h, (float4*)colsum, row4,
+                                                         d.G, total4);
+  *launches += 1;
+  return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;
+}
 
 static SelGeom sel_geom(const Dims& d) {
   SelGeom g;

@@ -141,5 +141,21 @@ __device__ __forceinline__ void colsum_chunk(const float* v, float c, const floa
   }
 }
 
+// Sweep 2 with one column sum per query head: the chunk's 32 rows in eight groups of four,
+// hs[i] = sum over rows 4i .. 4i+3 of 2^(c*s - b_r) (the caller adds the groups of a head).
+__device__ __forceinline__ void colsum_groups(const float* v, float c, const float* nb, float* hs) {
+  const float2 c2 = make_float2(c, c);
+  const float4* nb4 = reinterpret_cast<const float4*>(nb);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float4 bb = nb4[i];
+    const float2 e0 =
+        exp2_mufu_pair(__ffma2_rn(make_float2(v[4 * i], v[4 * i + 1]), c2, make_float2(bb.x, bb.y)));
+    const float2 e1 = exp2_mufu_pair(
+        __ffma2_rn(make_float2(v[4 * i + 2], v[4 * i + 3]), c2, make_float2(bb.z, bb.w)));
+    hs[i] = (e0.x + e0.y) + (e1.x + e1.y);
+  }
+}
+
 }  // namespace math
 }  // namespace laq

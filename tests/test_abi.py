@@ -33,8 +33,8 @@ def test_header_symbols_are_exported(binding):
 
 
 def test_struct_layout_and_version(binding):
-    assert ctypes.sizeof(binding.LaqParams) == 16 * 4 + 16 * 8 + 8
-    assert binding.LaqParams.q_stride_layer.offset == 64
+    assert ctypes.sizeof(binding.LaqParams) == 18 * 4 + 16 * 8 + 8
+    assert binding.LaqParams.q_stride_layer.offset == 72
     assert binding.laq_version() >= 100
     assert binding.status_string(0) == "ok"
     assert "argument" in binding.status_string(binding.LAQ_ERR_INVALID_ARG)

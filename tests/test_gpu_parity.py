@@ -28,21 +28,27 @@ def rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed, kscale=1.0):
     return q, k, v
 
 
-def run_evict(laq, q, k, v, R, kernel, B, local_window=0, pool_mode=0, score_mode=0, seq_lens=None):
+def run_evict(laq, q, k, v, R, kernel, B, local_window=0, pool_mode=0, score_mode=0, seq_lens=None,
+              group_mode=0):
     out = laq.evict(q.cuda(), k.cuda(), v.cuda(), B, pool_kernel=kernel, keep_tail=R,
                     want_scores=True, local_window=local_window, pool_mode=pool_mode,
-                    score_mode=score_mode, seq_lens=seq_lens)
+                    score_mode=score_mode, seq_lens=seq_lens, group_mode=group_mode)
     assert laq.laq_last_device_status(out["params"], out["ws"]) == laq.LAQ_OK
     return out
 
 
 def compare_all_units(laq, q, k, v, R, kernel, B, out=None, local_window=0, pool_mode=0,
-                      seq_lens=None):
+                      seq_lens=None, group_mode=0):
     """Full comparison of every unit of a (small) problem against the oracle."""
-    out = out or run_evict(laq, q, k, v, R, kernel, B, local_window, pool_mode, seq_lens=seq_lens)
+    out = out or run_evict(laq, q, k, v, R, kernel, B, local_window, pool_mode, seq_lens=seq_lens,
+                           group_mode=group_mode)
     ref = orc.evict(q, k, v, R, kernel, B, local_window=local_window, pool_mode=pool_mode,
-                    seq_lens=seq_lens)
+                    seq_lens=seq_lens, group_mode=group_mode)
     NL, Bt, Hkv, L = k.shape[0], k.shape[1], k.shape[2], k.shape[3]
+    if group_mode == 2:
+        # every query head is a unit of its own and gathers from its KV head
+        G = q.shape[2] // Hkv
+        k, v, Hkv = k.repeat_interleave(G, dim=2), v.repeat_interleave(G, dim=2), q.shape[2]
     got_scores = out["scores"].cpu().numpy()
     err = score_rel_err(got_scores, ref["scores"])
     assert err <= SCORE_RTOL, f"score rel err {err:.3e}"
@@ -592,6 +598,38 @@ def test_streaming_keep_set_and_its_compaction(laq):
     p = laq.params_for(q.cuda(), kd, W, 7, B, v=vd)
     assert laq.laq_streaming_indices(p, B + 1, idx, check=False) == laq.LAQ_ERR_INVALID_ARG
     assert laq.laq_streaming_indices(p, -1, idx, check=False) == laq.LAQ_ERR_INVALID_ARG
+
+
+GROUP_SHAPES = [
+    # NL Bt Hq Hkv D    L     W  k  B
+    (1, 2, 8, 2, 128, 1300, 32, 7, 120),   # one head per 32-row chunk (tensor-core path)
+    (2, 1, 8, 2, 128, 900, 8, 5, 64),      # four heads per chunk, M = 32
+    (1, 1, 8, 2, 128, 700, 16, 7, 90),     # two heads per chunk, M = 64
+    (1, 1, 4, 1, 128, 640, 64, 7, 100),    # a head spans two chunks, M = 256
+    (1, 1, 6, 2, 128, 500, 5, 3, 33),      # W = 5: heads straddle the groups of four -> CUDA-core path
+    (1, 1, 8, 2, 64, 400, 8, 7, 60),       # head_dim 64: CUDA-core path
+]
+
+
+@pytest.mark.parametrize("mode", [1, 2], ids=["max-over-group", "per-query-head"])
+@pytest.mark.parametrize("shape", GROUP_SHAPES, ids=[f"L{s[5]}-W{s[6]}-G{s[2] // s[3]}-D{s[4]}" for s in GROUP_SHAPES])
+def test_group_modes_match_oracle(laq, shape, mode):
+    NL, Bt, Hq, Hkv, D, L, W, kernel, B = shape
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=300 + L + mode, kscale=1.5)
+    err, _ = compare_all_units(laq, q, k, v, W, kernel, B, group_mode=mode)
+    assert err < SCORE_RTOL
+
+
+def test_group_modes_with_ragged_prompts_and_raw_mode_refusal(laq):
+    NL, Bt, Hq, Hkv, D, L, W, kernel, B = 1, 3, 8, 2, 128, 1000, 16, 7, 80
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=311, kscale=1.5)
+    k[:, 1, :, 600:] = float("nan")   # never read
+    k[:, 2, :, 81:] = float("nan")
+    for mode in (1, 2):
+        compare_all_units(laq, q, k, v, W, kernel, B, seq_lens=[1000, 600, 81], group_mode=mode)
+    p = laq.params_for(q.cuda(), k.cuda(), W, kernel, B)
+    p.group_mode, p.score_mode = laq.LAQ_GROUP_MAX, laq.LAQ_SCORE_RAW
+    assert laq.laq_workspace_bytes(p) == 0   # an unsupported combination has no workspace size
 
 
 def test_config1_full_with_planted_key(laq):
