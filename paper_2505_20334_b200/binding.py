@@ -67,12 +67,13 @@ class LaqError(RuntimeError):
         super().__init__(f"{where}: {status_string(status)} (laq_status {status})")
 
 
-def _load() -> ctypes.CDLL:
-    if not os.path.exists(LIB_PATH):
+def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
+    """Loads a build of the library and declares the argument types of its entry points."""
+    if not os.path.exists(path):
         raise ImportError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2505_20334_b200.build` "
+            f"{path} is missing: build it with `python -m paper_2505_20334_b200.build` "
             "(there is no fallback path)")
-    lib = ctypes.CDLL(LIB_PATH)
+    lib = ctypes.CDLL(path)
     vp, sz, pp = ctypes.c_void_p, ctypes.c_size_t, ctypes.POINTER(LaqParams)
     lib.laq_params_dense_strides.argtypes = [pp]
     lib.laq_params_dense_strides.restype = None
@@ -117,7 +118,7 @@ def _load() -> ctypes.CDLL:
     return lib
 
 
-lib = _load()
+lib = load_library()
 
 
 def status_string(status: int) -> str:

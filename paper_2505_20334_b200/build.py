@@ -34,18 +34,25 @@ def _deps_mtime():
     return max(os.path.getmtime(f) for f in files)
 
 
-def build_liblaq(force: bool = False, verbose: bool = False, defines=()) -> str:
+def build_liblaq(force: bool = False, verbose: bool = False, defines=(), variant: str = "") -> str:
     """Compiles liblaq.so if it is missing or older than its sources. `defines` are extra
-    ``-DNAME=VALUE`` strings for tuning builds (they force a rebuild)."""
-    force = force or bool(defines)
-    if not force and os.path.exists(LIB_PATH) and os.path.getmtime(LIB_PATH) >= _deps_mtime():
-        return LIB_PATH
-    os.makedirs(OBJ_DIR, exist_ok=True)
+    ``-DNAME=VALUE`` strings for tuning builds (they force a rebuild). A non-empty `variant` builds
+    ``_build/<variant>/liblaq_<variant>.so`` from the same sources with those defines and leaves
+    liblaq.so alone (the tests use it for a copy of the library with test hooks compiled in)."""
+    lib_path, obj_dir = LIB_PATH, OBJ_DIR
+    if variant:
+        obj_dir = os.path.join(OBJ_DIR, variant)
+        lib_path = os.path.join(obj_dir, f"liblaq_{variant}.so")
+    else:
+        force = force or bool(defines)
+    if not force and os.path.exists(lib_path) and os.path.getmtime(lib_path) >= _deps_mtime():
+        return lib_path
+    os.makedirs(obj_dir, exist_ok=True)
     nvcc = os.environ.get("NVCC", "nvcc")
     extra = ["-Xptxas", "-v"] if verbose else []
 
     def compile_one(src):
-        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
+        obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
         cmd = [nvcc, *NVCC_FLAGS, *extra, *defines, "-c", src, "-o", obj]
         r = subprocess.run(cmd, capture_output=True, text=True)
         return obj, r
@@ -58,12 +65,12 @@ def build_liblaq(force: bool = False, verbose: bool = False, defines=()) -> str:
             if r.returncode != 0:
                 raise RuntimeError(f"nvcc failed for {obj}")
             objs.append(obj)
-    link = [nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB_PATH, *objs]
+    link = [nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", lib_path, *objs]
     r = subprocess.run(link, capture_output=True, text=True)
     if r.returncode != 0:
         sys.stderr.write(r.stdout + r.stderr)
         raise RuntimeError("link of liblaq.so failed")
-    return LIB_PATH
+    return lib_path
 
 
 if __name__ == "__main__":

@@ -60,7 +60,12 @@ constexpr int kMaxSlots = 4;  // K stages in shared memory = TMEM accumulator bu
 constexpr int kStatSlots = 3;
 constexpr uint32_t kKStageBytes = TILE_KEYS * 128 * 2;  // 128 keys x 128 dims x bf16
 constexpr uint32_t kCtlBytes = 34816;
-constexpr long long kTimeoutCycles = 4000000000LL;  // ~2 s: every device-side wait gives up after this
+#ifndef LAQ_TIMEOUT_CYCLES
+#define LAQ_TIMEOUT_CYCLES 4000000000LL  // ~2 s: every device-side wait gives up after this
+#endif
+constexpr long long kTimeoutCycles = LAQ_TIMEOUT_CYCLES;
+// after a wait has run out: how long a role waits for its own asynchronous work before it leaves
+constexpr long long kDrainCycles = 2000000LL;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kMaxDevices = 64;
 // two MMA lanes, statistics-out warp, statistics-in warps, softmax warps
@@ -84,6 +89,7 @@ struct TcArgs {
   int tasks_per_layer;  // per-prompt lengths: sweep-1 tasks of one layer (all prompts and KV heads)
   uint32_t total_tickets;
   float scale_log2;
+  int64_t withhold_unit;  // test hook: this unit's statistics are never published (-1: none)
   int32_t* hdr;
   int32_t* cnt;
   float2* part;
@@ -112,6 +118,7 @@ struct Ctl {
   // t - 5, and the pair waiting for tile t then sees a stale phase (seen as a wait that ran out).
   uint64_t mma_done[kMaxSlots];
   uint64_t tmem_empty[kMaxSlots];
+  uint64_t drain[2];  // one per MMA issuer: completion of everything it has issued (abort path)
   uint64_t task_full[kTaskSlots], task_empty[kTaskSlots];
   uint64_t stat_full[kStatSlots], stat_empty[kStatSlots];
   uint64_t boff_full[kStatSlots], boff_empty[kStatSlots];
@@ -289,6 +296,14 @@ __device__ __forceinline__ bool mbar_wait(const TcArgs& a, Ctl* ctl, uint32_t ba
     }
   }
   return true;
+}
+
+// Waits for a barrier after the CTA has given up (abort is set, so mbar_wait would return at
+// once): a short, bounded wait for asynchronous work of this thread's own that is still in flight.
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
+  while (!mbar_try_wait_for(bar, parity, 1000) && clock64() - t0 < kDrainCycles) {
+  }
 }
 
 __device__ __forceinline__ int ld_acquire(const int32_t* p) {
@@ -472,6 +487,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       mbar_init(smem_u32(&ctl->mma_done[i]), 1);
       mbar_init(smem_u32(&ctl->tmem_empty[i]), 8);  // the 8 warps of one warpgroup pair
     }
+    mbar_init(smem_u32(&ctl->drain[0]), 1);
+    mbar_init(smem_u32(&ctl->drain[1]), 1);
     for (int i = 0; i < kTaskSlots; ++i) {
       mbar_init(smem_u32(&ctl->task_full[i]), 1);
       mbar_init(smem_u32(&ctl->task_empty[i]), kTaskConsumers);
@@ -577,9 +594,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         task = next;
       }
       if (ctl->abort) {
-        // give loads that are still in flight time to land before the CTA exits
-        const long long t0 = clock64();
-        while (clock64() - t0 < 200000) __nanosleep(256);
+        // A wait ran out somewhere in this CTA. Loads that this lane has requested may still be
+        // on their way into shared memory: wait (bounded) for the full-barrier of every K stage
+        // and Q stage armed last, so that nothing is written into the CTA's memory after it exits.
+        const uint32_t n_slots = slot_mask + 1u;
+        for (uint32_t t = kcount > n_slots ? kcount - n_slots : 0u; t < kcount; ++t)
+          mbar_drain(smem_u32(&ctl->k_full[t & slot_mask]), (t >> kSlotShift) & 1u);
+        for (uint32_t t = qcount > 2u ? qcount - 2u : 0u; t < qcount; ++t)
+          mbar_drain(smem_u32(&ctl->q_full[t & 1u]), (t >> 1) & 1u);
       }
     }
   } else if (warp == 1 || warp == kMmaWarpB) {
@@ -641,6 +663,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         umma_commit(smem_u32(&ctl->q_empty[qs]));
         ++qc;
       }
+      if (ctl->abort) {
+        // MMAs this lane has issued may still be running: one more commit tracks all of them, and
+        // the (bounded) wait for it ends before tensor memory is given back at the end of the kernel
+        umma_commit(smem_u32(&ctl->drain[issuer]));
+        mbar_drain(smem_u32(&ctl->drain[issuer]), 0u);
+      }
     }
   } else if (warp == 2) {
     // ================= statistics out =================
@@ -677,7 +705,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       __syncwarp();
       if (lane == 0) {
         mbar_arrive(smem_u32(&ctl->stat_empty[s]));
-        atomicAdd(&a.cnt[task.unit], 1);
+        if (task.unit != a.withhold_unit) atomicAdd(&a.cnt[task.unit], 1);
       }
       ++sc;
     }
@@ -704,7 +732,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
           uint32_t spins = 0;
           while (ld_acquire(ctr) < n_partials) {
             if ((++spins & 15u) == 0) {
-              if (ctl->abort) { ready = 0; break; }
+              // another CTA has already given up: do not wait out a limit of our own
+              if (ctl->abort || ld_acquire(&a.hdr[HDR_STATUS]) != 0) {
+                ctl->abort = 1;
+                ready = 0;
+                break;
+              }
               if (clock64() - t0 > kTimeoutCycles) { record_timeout(a, ctl, 42); ready = 0; break; }
             }
             __nanosleep(32);
@@ -965,8 +998,25 @@ bool make_map(CUtensorMap* map, const void* base, const uint64_t dims[5], const 
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-}  // namespace
+#ifdef LAQ_TEST_HOOKS
+std::atomic<long long> g_withhold_unit{-1};
+int64_t test_withhold_unit() { return g_withhold_unit.load(); }
+#else
+int64_t test_withhold_unit() { return -1; }
+#endif
 
+}  // namespace
+}  // namespace laq
+
+#ifdef LAQ_TEST_HOOKS
+// Test builds only (never part of liblaq.so): the scoring kernel withholds the statistics of one
+// unit, so that the bounded wait of that unit's second sweep runs out. -1 switches it off.
+extern "C" __attribute__((visibility("default"))) void laq_test_withhold_unit(long long unit) {
+  laq::g_withhold_unit.store(unit);
+}
+#endif
+
+namespace laq {
 laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& w, const void* q,
                            const void* k, char* ws, cudaStream_t stream, int* launches) {
   TcArgs a;
@@ -1028,6 +1078,7 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   a.part = (float2*)(ws + w.off_part);
   a.colsum = (float*)(ws + (d.group_mode != LAQ_GROUP_SUM ? w.off_colsum_h : w.off_colsum));
   a.sl = d.sl;
+  a.withhold_unit = test_withhold_unit();
   const bool wide = d.M > 128;
   const int q_rows = wide ? 256 : 128, n_slots = wide ? 2 : 4;
   const bool dup = w.M_pad <= 64;  // sweep 1 holds every query row twice, on lanes r and 64 + r
