@@ -254,27 +254,6 @@ __device__ __forceinline__ void tmem_ld_wait(float* v) {
                :
                : "memory");
 }
-// The same for 16 columns.
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
-  uint32_t* r = reinterpret_cast<uint32_t*>(v);
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
-        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
-        "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait16(float* v) {
-  uint32_t* r = reinterpret_cast<uint32_t*>(v);
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]),
-                 "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]),
-                 "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
-               :
-               : "memory");
-}
 // Adds to a global fp32 without returning a value.
 __device__ __forceinline__ void red_add(float* p, float v) {
   asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
@@ -459,41 +438,6 @@ __device__ __forceinline__ void stats_cols64(uint32_t taddr, float c, float& m, 
   stats_chunk<kPoly>(v, c, m, l);
 }
 
-// Sweep 1 for units of at most 16 rows (one or two lookahead steps, Section 6.2): the tile is
-// produced with the keys on the TMEM lanes, as in sweep 2, so that the MMA is 128 x 16 instead of
-// 128 x 128 with 112 padding rows. This thread owns key `key` and holds the tile's 16 logits of
-// that key in v; ref[r] / acc[r] are the warp's reference shift of row r (the same in all lanes)
-// and this lane's part of the row sum. A value far above a reference shows as a huge exponential:
-// the warp then raises the references of all rows to the largest logit it holds and rescales.
-// Row r sees keys below vis_of(r) only (a causal local query, or the end of the prompt).
-template <typename VisOf>
-__device__ __forceinline__ void stats_keys16(const float* v, float c, int key, bool plain, VisOf vis_of,
-                                             float* ref, float* acc) {
-  float e[16];
-  float big = 0.f;
-#pragma unroll
-  for (int r = 0; r < 16; ++r) {
-    e[r] = ex2(fmaf(v[r], c, -ref[r]));
-    if (!plain && key >= vis_of(r)) e[r] = 0.f;
-    big = fmaxf(big, e[r]);
-  }
-  if (__any_sync(0xffffffffu, !(big < kChunkSumLimit))) {
-#pragma unroll
-    for (int r = 0; r < 16; ++r) {
-      const float t = (plain || key < vis_of(r)) ? v[r] * c : -3.0e38f;
-      float mx = t;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-      const float m_new = fmaxf(ref[r], mx);
-      acc[r] *= ex2(ref[r] - m_new);
-      ref[r] = m_new;
-      e[r] = ex2(t - m_new);
-    }
-  }
-#pragma unroll
-  for (int r = 0; r < 16; ++r) acc[r] += e[r];
-}
-
 // ------------------------------------------------------------------ the kernel
 // kDup: M <= 64, sweep 1 holds every query row twice (on TMEM lanes r and 64 + r).
 // kWide: 128 < M <= 256, two row blocks per tile, so an accumulator buffer takes 256 TMEM columns
@@ -501,8 +445,7 @@ __device__ __forceinline__ void stats_keys16(const float* v, float c, int key, b
 // kPerHead: sweep 2 keeps one column sum per query head (colsum is [U*G][L_pad]); the launcher
 // only picks it when a head's rows never straddle a group of four rows or a 32-row chunk unevenly
 // (W a multiple of 4 that divides 32, or 32 or 64).
-// kNarrow: M <= 16; sweep 1 runs with the keys on the TMEM lanes (see stats_keys16).
-template <bool kDup, bool kWide, bool kPerHead, bool kNarrow>
+template <bool kDup, bool kWide, bool kPerHead>
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
                 const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ TcArgs a) {
@@ -671,7 +614,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
     if (lane == 0) {
       const uint32_t issuer = warp == 1 ? 0u : 1u;
       uint32_t tc_base = 0, my_next = issuer, qc = 0, tk = 0;
-      const uint32_t idesc_s1 = kNarrow ? instr_desc(128, 16) : instr_desc(128, TILE_KEYS);
+      const uint32_t idesc_s1 = instr_desc(128, TILE_KEYS);
       const uint32_t idesc_s2 = instr_desc(128, a.M_pad);
       const uint32_t q_half16 = kQRows * 8u;  // (q_rows * 128 bytes) >> 4
       const uint32_t k_lo0 = smem_desc_lo(k_base), q_lo0 = smem_desc_lo(q_base);
@@ -697,7 +640,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
           const uint32_t k_lo = k_lo0 + s * (kKStageBytes >> 4);
           const uint32_t d_tmem = tmem_base + s * kTbCols;
           // k-step kk covers dims [16 kk, 16 kk + 16): 32 bytes inside the 64-dim half (kk >> 2)
-          if (task.sweep == 0 && !kNarrow) {
+          if (task.sweep == 0) {
             for (int rb = 0; rb < RB; ++rb) {
 #pragma unroll
               for (int kk = 0; kk < 8; ++kk)
@@ -710,8 +653,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk)
               umma_bf16(d_tmem, k_lo + (kk >> 2) * (kKStageBytes >> 5) + (kk & 3) * 2u,
-                        q_lo + (kk >> 2) * q_half16 + (kk & 3) * 2u, kSmemDescHi,
-                        task.sweep == 0 ? idesc_s1 : idesc_s2, kk > 0);
+                        q_lo + (kk >> 2) * q_half16 + (kk & 3) * 2u, kSmemDescHi, idesc_s2, kk > 0);
           }
           umma_commit(smem_u32(&ctl->mma_done[s]));
         }
@@ -751,15 +693,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       float2* dst = a.part + ((int64_t)task.unit * a.n_part + task.chunk) * a.M_pad;
       for (int row = lane; row < a.M_pad; row += 32) {
         float m = -1e30f, l = 0.f;
-        if (kNarrow) {
-          // one (shift, sum) per row from every warp of the two warpgroups that took tiles
-          if (row < 16) {
-#pragma unroll
-            for (int wq = 0; wq < 8; ++wq) merge_stat(m, l, ctl->stat[s][(wq >> 2) * 2][(wq & 3) * 16 + row]);
-          }
-          dst[row] = make_float2(m, l);
-          continue;
-        }
 #pragma unroll
         for (int g = 0; g < kSoftmaxWgs; ++g) merge_stat(m, l, ctl->stat[s][g][row]);
         if (kDup) {  // the second copy of the row saw the other key columns
@@ -881,12 +814,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
       const int vis0 = qi0 < a.W_local ? Lu - a.W_local + qi0 + 1 : Lu;
       const int vis1 = qi1 < a.W_local ? Lu - a.W_local + qi1 + 1 : Lu;
       float m0 = -1e30f, l0 = 0.f, m1 = -1e30f, l1 = 0.f;
-      float nref[kNarrow ? 16 : 1], nacc[kNarrow ? 16 : 1];  // sweep 1 with the keys on the lanes
-#pragma unroll
-      for (int r = 0; r < (kNarrow ? 16 : 1); ++r) {
-        nref[r] = -1e30f;
-        nacc[r] = 0.f;
-      }
       const float* nboff = nullptr;
       const float* nbsat = nullptr;
       if (task.sweep == 1) {
@@ -909,19 +836,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         const uint32_t taddr = lane_addr + s * kTbCols;
         const uint32_t empty_bar = smem_u32(&ctl->tmem_empty[s]);
         float v[32];
-        if (kNarrow && task.sweep == 0) {
-          if (half == 1) {
-            release_buffer(empty_bar, lane);  // 16 columns: the first warpgroup of the pair takes them
-          } else {
-            tmem_ld16(taddr, v);
-            tmem_ld_wait16(v);
-            release_buffer(empty_bar, lane);
-            const int W = a.W, Wl = a.W_local;
-            stats_keys16(v, c, key0 + row_in_wg, key0 + TILE_KEYS <= Lu - Wl,
-                         [=](int r) { const int qi = r % W; return qi < Wl ? Lu - Wl + qi + 1 : Lu; },
-                         nref, nacc);
-          }
-        } else if (task.sweep == 0) {
+        if (task.sweep == 0) {
           const int valid = min(TILE_KEYS, Lu - key0);
           // row blocks beyond the unit's rows are skipped (warp-uniform)
           const bool rows0 = (kDup ? (quad & 1) : quad) * 32 < a.M;
@@ -1015,20 +930,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
         // hand this warpgroup's statistics to the statistics-out warp
         const uint32_t s = s1c % kStatSlots;
         if (!mbar_wait(a, ctl, smem_u32(&ctl->stat_empty[s]), ((s1c / kStatSlots) & 1u) ^ 1u, 23)) break;
-        if (kNarrow) {
-          if (half == 0) {
-#pragma unroll
-            for (int r = 0; r < 16; ++r) {
-              float sum = nacc[r];
-#pragma unroll
-              for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-              if (lane == r) ctl->stat[s][wg][quad * 16 + r] = make_float2(nref[r], sum);
-            }
-          }
-        } else {
-          ctl->stat[s][wg][row_in_wg] = make_float2(m0, l0);
-          ctl->stat[s][wg][128 + row_in_wg] = make_float2(m1, l1);
-        }
+        ctl->stat[s][wg][row_in_wg] = make_float2(m0, l0);
+        ctl->stat[s][wg][128 + row_in_wg] = make_float2(m1, l1);
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctl->stat_full[s]));
         ++s1c;
@@ -1178,9 +1081,7 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
   a.withhold_unit = test_withhold_unit();
   const bool wide = d.M > 128;
   const int q_rows = wide ? 256 : 128, n_slots = wide ? 2 : 4;
-  const bool per_head = d.group_mode != LAQ_GROUP_SUM;
-  const bool narrow = d.M <= 16 && !per_head;  // sweep 1 with the keys on the TMEM lanes
-  const bool dup = w.M_pad <= 64 && !narrow;   // sweep 1 holds every query row twice, on lanes r and 64 + r
+  const bool dup = w.M_pad <= 64;  // sweep 1 holds every query row twice, on lanes r and 64 + r
 
   CUtensorMap tmap_q, tmap_k;
   const uint64_t qdims[5] = {128, (uint64_t)d.W, (uint64_t)d.Hq, (uint64_t)d.Bt, (uint64_t)d.NL};
@@ -1193,16 +1094,16 @@ laq_status score_tc_launch(const laq_params& p, const Dims& d, const Workspace& 
     return score_simt_launch(p, d, w, q, k, ws, stream, launches);  // layout TMA cannot describe
 
   const size_t smem = kCtlBytes + 2u * (size_t)q_rows * 256u + (size_t)n_slots * kKStageBytes;
-  auto kernel = narrow     ? score_tc_kernel<false, false, false, true>
-                : per_head ? (dup ? score_tc_kernel<true, false, true, false>
-                                  : (wide ? score_tc_kernel<false, true, true, false>
-                                          : score_tc_kernel<false, false, true, false>))
-                           : (dup ? score_tc_kernel<true, false, false, false>
-                                  : (wide ? score_tc_kernel<false, true, false, false>
-                                          : score_tc_kernel<false, false, false, false>));
+  const bool per_head = d.group_mode != LAQ_GROUP_SUM;
+  auto kernel = per_head ? (dup ? score_tc_kernel<true, false, true>
+                                : (wide ? score_tc_kernel<false, true, true>
+                                        : score_tc_kernel<false, false, true>))
+                         : (dup ? score_tc_kernel<true, false, false>
+                                : (wide ? score_tc_kernel<false, true, false>
+                                        : score_tc_kernel<false, false, false>));
   // the shared-memory opt-in is a per-device attribute of each kernel variant: set once
   static std::atomic<uint32_t> smem_opted_in[kMaxDevices];
-  const uint32_t variant_bit = narrow ? 1u << 6 : 1u << ((dup ? 0 : (wide ? 1 : 2)) + (per_head ? 3 : 0));
+  const uint32_t variant_bit = 1u << ((dup ? 0 : (wide ? 1 : 2)) + (per_head ? 3 : 0));
   if (dev >= kMaxDevices || !(smem_opted_in[dev].load(std::memory_order_acquire) & variant_bit)) {
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)

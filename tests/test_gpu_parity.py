@@ -84,9 +84,9 @@ SHAPES = [
     (1, 1, 4, 2, 128, 50, 4, 7, 20),       # L smaller than one tile
     (1, 1, 8, 2, 64, 500, 8, 7, 90),       # head_dim 64: CUDA-core path
     (1, 1, 4, 1, 256, 260, 8, 5, 48),      # head_dim 256: CUDA-core path
-    (2, 2, 8, 2, 128, 4500, 1, 7, 64),     # one lookahead step: M = 4, keys on the lanes in both sweeps
+    (2, 2, 8, 2, 128, 4500, 1, 7, 64),     # one lookahead step (Section 6.2): M = 4
     (1, 1, 8, 2, 128, 2500, 2, 5, 40),     # two lookahead steps: M = 8
-    (1, 1, 16, 2, 128, 1100, 2, 3, 50),    # M = 16, the widest unit of that path
+    (1, 1, 16, 2, 128, 1100, 2, 3, 50),    # M = 16
 ]
 
 
@@ -518,8 +518,8 @@ def test_extreme_logits_and_late_maximum(laq):
 
 
 def test_extreme_logits_with_one_or_two_lookahead_steps(laq):
-    # the same stress for units of at most 16 rows, whose statistics sweep keeps one reference per
-    # row and warp: the large key arrives late, after many tiles of small logits
+    # the same stress for the short windows of Section 6.2 (one or two lookahead steps, M = 8):
+    # the large key arrives late, after many tiles of small logits
     NL, Bt, Hq, Hkv, D, L, W, kernel, B = 1, 1, 8, 2, 128, 4200, 2, 7, 90
     g = torch.Generator().manual_seed(405)
     q = torch.randn((NL, Bt, Hq, W, D), generator=g).to(torch.bfloat16)
