@@ -652,6 +652,51 @@ def test_group_modes_with_ragged_prompts_and_raw_mode_refusal(laq):
     assert laq.laq_workspace_bytes(p) == 0   # an unsupported combination has no workspace size
 
 
+def test_per_layer_budgets_with_per_query_head_selection(laq):
+    # the two options together: the ragged pool then holds [Bt][Hq][B_n] entries per layer
+    NL, Bt, Hq, Hkv, D, L, W, kernel = 3, 1, 4, 2, 128, 900, 8, 5
+    budgets = [40, 120, 64]
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=73, kscale=1.5)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    p = laq.params_for(qd, kd, W, kernel, max(budgets), v=vd)
+    p.group_mode = laq.LAQ_GROUP_PER_HEAD
+    entries = laq.laq_layers_pool_entries(p, budgets)
+    assert entries == Bt * Hq * sum(budgets)
+    idx = torch.empty(entries, dtype=torch.int32, device="cuda")
+    k_out = torch.empty((entries, D), dtype=torch.bfloat16, device="cuda")
+    v_out = torch.empty_like(k_out)
+    ws = laq.alloc_workspace(p, "cuda")
+    laq.laq_evict_layers(p, budgets, qd, kd, vd, k_out, v_out, idx, None, ws)
+    assert laq.laq_last_device_status(p, ws) == laq.LAQ_OK
+    ref = orc.evict_layers(q, k, v, W, kernel, budgets, group_mode=2)
+    got = idx.cpu().numpy()
+    G, row = Hq // Hkv, 0
+    for n, B in enumerate(budgets):
+        for hq in range(Hq):
+            gi = got[row:row + B]
+            check_index_set(gi, ref["idx"][row:row + B], ref["scores"][n, 0, hq], L, W, B)
+            assert (bits(k_out[row:row + B]) == bits(k[n, 0, hq // G])[gi]).all()
+            assert (bits(v_out[row:row + B]) == bits(v[n, 0, hq // G])[gi]).all()
+            row += B
+
+
+def test_gather_of_more_units_than_one_grid_dimension_holds(laq):
+    # 70 000 units: the gather runs in slabs of 65 535 units
+    NL, Bt, Hkv, D, L, B = 1, 8750, 8, 8, 16, 4
+    g = torch.Generator().manual_seed(74)
+    k = torch.randn((NL, Bt, Hkv, L, D), generator=g).to(torch.bfloat16).cuda()
+    v = torch.randn((NL, Bt, Hkv, L, D), generator=g).to(torch.bfloat16).cuda()
+    idx = torch.stack([torch.randperm(L, generator=g)[:B].sort().values for _ in range(64)])
+    idx = idx.repeat(NL * Bt * Hkv // 64 + 1, 1)[:NL * Bt * Hkv].view(NL, Bt, Hkv, B).to(torch.int32).cuda()
+    p = laq.make_params(NL, Bt, Hkv, Hkv, D, L, 1, 1, 1, B)
+    k_out = torch.zeros((NL, Bt, Hkv, B, D), dtype=torch.bfloat16, device="cuda")
+    v_out = torch.zeros_like(k_out)
+    laq.laq_compact(p, k, v, idx, k_out, v_out)
+    want_k = torch.gather(k, 3, idx.long()[..., None].expand(-1, -1, -1, -1, D))
+    want_v = torch.gather(v, 3, idx.long()[..., None].expand(-1, -1, -1, -1, D))
+    assert torch.equal(k_out, want_k) and torch.equal(v_out, want_v)
+
+
 def test_config1_full_with_planted_key(laq):
     cfg = synth.CONFIGS[1]
     inp = synth.make_inputs(cfg, "cpu")
