@@ -228,30 +228,56 @@ __device__ __forceinline__ void transpose32(uint32_t (&a)[32]) {
 // kPoolStatic > 0 fixes the pooling kernel at compile time (unrolled taps); 0 takes it from `kpool`.
 // kThreads: block size (128 .. 1024); a unit of up to 32 * kThreads scored positions takes the
 // smallest one, so that several blocks of short units share an SM.
-template <int kPoolStatic, int kThreads>
+// kPair: a unit of up to 65536 scored positions is taken by a cluster of two 1024-thread CTAs,
+// CTA r holding positions [32768 r, 32768 r + 32768) in registers as before. What the threshold
+// search needs from the other half is one count per bit step, read from the peer's shared memory
+// after a cluster barrier; the kept positions of the second half are written behind those of the
+// first. Both CTAs execute the same barriers whatever their data, so neither can be left waiting.
+constexpr int kPairHalf = kRegItems * 1024;  // positions per CTA of a pair
+constexpr int kPairHalo = 4;                 // staged positions on either side of a half (>= kpool / 2)
+
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Reads the 32-bit word at the same shared-memory address in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t ld_peer_u32(const uint32_t* p, uint32_t rank) {
+  const uint32_t local = (uint32_t)__cvta_generic_to_shared(p);
+  uint32_t remote, v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
+  asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(remote) : "memory");
+  return v;
+}
+
+template <int kPoolStatic, int kThreads, bool kPair>
 __global__ void __launch_bounds__(kThreads, 1024 / kThreads) pool_select_reg_kernel(
     const float* __restrict__ colsum, int L_pad, float* pooled_out, int32_t* __restrict__ idx,
     int kpool, float inv_k, int pool_max, const __grid_constant__ SelGeom g) {
   constexpr int kWarps = kThreads / 32;
   __shared__ uint32_t s_cnt[2][kWarps];
   __shared__ uint32_t s_gt[kWarps], s_eq[kWarps];
+  __shared__ uint32_t s_x[2], s_tot[2];  // pair: this CTA's count of the current bit step; its totals
   extern __shared__ __align__(16) float s_c[];  // the unit's column sums, [0, Ls) rounded up to 4
-  const int64_t u = blockIdx.x;
+  const uint32_t rank = kPair ? (blockIdx.x & 1u) : 0u;  // cluster of (2, 1, 1): rank = blockIdx.x % 2
+  const int64_t u = kPair ? (int64_t)(blockIdx.x >> 1) : (int64_t)blockIdx.x;
   const int Ls = unit_scored(g, u), Kb = unit_kb(g, u), R = g.R;
   int32_t* out = unit_out(g, idx, u);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int pos0 = kPair ? (int)rank * kPairHalf : 0;  // first position this CTA holds
   // One coalesced pass brings the column sums on chip (rows are 512-byte aligned and padded to
   // a multiple of 128 floats); the pooling taps then read shared memory instead of L1/L2.
+  // A CTA of a pair stages its half and a halo of kPairHalo positions on either side.
+  const int c_lo = kPair ? max(0, pos0 - kPairHalo) : 0;
+  const int c_hi = kPair ? min(Ls, pos0 + kPairHalf + kPairHalo) : Ls;
   {
-    const float4* src = reinterpret_cast<const float4*>(colsum + u * (int64_t)L_pad);
+    const float4* src = reinterpret_cast<const float4*>(colsum + u * (int64_t)L_pad + c_lo);
     float4* dst = reinterpret_cast<float4*>(s_c);
-    const int n4 = (Ls + 3) >> 2;
+    const int n4 = (max(0, c_hi - c_lo) + 3) >> 2;
 #pragma unroll 8
     for (int k = tid; k < n4; k += kThreads) dst[k] = __ldcs(src + k);
   }
   __syncthreads();
-  const float* c = s_c;
-  const int base = warp * (kRegItems * 32) + lane;
+  const float* c = s_c - c_lo;  // indexed by position
+  const int base = pos0 + warp * (kRegItems * 32) + lane;
   const int h = (kPoolStatic > 0 ? kPoolStatic : kpool) / 2;
 
   uint32_t w[kRegItems];  // first the keys, then their bit planes
@@ -298,7 +324,14 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads) pool_select_reg_ker
     uint32_t* slot = s_cnt[bit & 1];
     if (lane == 0) slot[warp] = n_warp;
     __syncthreads();
-    const uint32_t n = __reduce_add_sync(0xffffffffu, lane < kWarps ? slot[lane] : 0u);
+    uint32_t n = __reduce_add_sync(0xffffffffu, lane < kWarps ? slot[lane] : 0u);
+    if (kPair) {
+      // add the other half's count of this step (the two slots alternate: a slot is rewritten
+      // only after the peer has passed the next barrier, i.e. after it has read it)
+      if (tid == 0) s_x[bit & 1] = n;
+      cluster_sync_all();
+      n += ld_peer_u32(&s_x[bit & 1], rank ^ 1u);
+    }
     if (above + n >= (uint32_t)Kb) {
       theta |= 1u << bit;
       alive = ones;
@@ -324,6 +357,23 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads) pool_select_reg_ker
     gt_run += s_gt[ww];
     eq_run += s_eq[ww];
   }
+  if (kPair) {
+    // the second half writes behind the first: its running counts start from the first half's totals
+    if (tid == 0) {
+      uint32_t tg = 0, te = 0;
+      for (int ww = 0; ww < kWarps; ++ww) {
+        tg += s_gt[ww];
+        te += s_eq[ww];
+      }
+      s_tot[0] = tg;
+      s_tot[1] = te;
+    }
+    cluster_sync_all();
+    if (rank == 1u) {
+      gt_run += ld_peer_u32(&s_tot[0], 0u);
+      eq_run += ld_peer_u32(&s_tot[1], 0u);
+    }
+  }
   const uint32_t lt_mask = (1u << lane) - 1u;
 #pragma unroll
   for (int it = 0; it < kRegItems; ++it) {
@@ -337,7 +387,9 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads) pool_select_reg_ker
     gt_run += __popc(bg);
     eq_run += __popc(be);
   }
-  for (int t = tid; t < R; t += kThreads) out[Kb + t] = Ls + t;
+  if (rank == 0u)
+    for (int t = tid; t < R; t += kThreads) out[Kb + t] = Ls + t;
+  if (kPair) cluster_sync_all();  // no CTA leaves while its peer may still read its shared memory
 }
 
 // c[u][j] = max over the G heads of c_h[u*G + g][j] (LAQ_GROUP_MAX); rows are L_pad floats,
@@ -413,11 +465,11 @@ laq_status pool_select_launch(const Dims& d, const float* colsum, int L_pad, flo
     const int threads = d.Ls <= 32 * 128 ? 128 : (d.Ls <= 32 * 256 ? 256 : (d.Ls <= 32 * 512 ? 512 : 1024));
 #define LAQ_LAUNCH_POOL_SELECT_T(KP, T)                                                               \
   {                                                                                                   \
-    if (cudaFuncSetAttribute(pool_select_reg_kernel<KP, T>,                                           \
+    if (cudaFuncSetAttribute(pool_select_reg_kernel<KP, T, false>,                                    \
                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_c) != cudaSuccess) \
       return LAQ_ERR_CUDA;                                                                            \
-    pool_select_reg_kernel<KP, T><<<grid, T, smem_c, stream>>>(colsum, L_pad, pooled_out, idx, d.kpool, \
-                                                               inv_k, d.pool_max, g);                 \
+    pool_select_reg_kernel<KP, T, false><<<grid, T, smem_c, stream>>>(colsum, L_pad, pooled_out, idx, \
+                                                                      d.kpool, inv_k, d.pool_max, g); \
   }
 #define LAQ_LAUNCH_POOL_SELECT(KP)                     \
   switch (threads) {                                   \
@@ -438,6 +490,43 @@ laq_status pool_select_launch(const Dims& d, const float* colsum, int L_pad, flo
     *launches += 1;
     *done = true;
     return cudaGetLastError() == cudaSuccess ? LAQ_OK : LAQ_ERR_CUDA;
+  }
+  if (d.Ls <= 2 * kPairHalf && d.kpool / 2 <= kPairHalo && d.U <= 0x3fffffff) {
+    // two CTAs per unit, as a cluster: each holds half of the positions in registers
+    const float inv_k = 1.0f / (float)d.kpool;
+    const size_t smem_c = (size_t)(kPairHalf + 2 * kPairHalo) * sizeof(float);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * d.U));
+    cfg.blockDim = dim3(1024);
+    cfg.dynamicSmemBytes = smem_c;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int kpool = d.kpool, pool_max = d.pool_max;
+#define LAQ_LAUNCH_POOL_SELECT_PAIR(KP)                                                              \
+  {                                                                                                  \
+    if (cudaFuncSetAttribute(pool_select_reg_kernel<KP, 1024, true>,                                 \
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_c) != cudaSuccess || \
+        cudaLaunchKernelEx(&cfg, pool_select_reg_kernel<KP, 1024, true>, colsum, L_pad, pooled_out,  \
+                           idx, kpool, inv_k, pool_max, g) != cudaSuccess)                           \
+      return LAQ_ERR_CUDA;                                                                           \
+  }
+    switch (d.kpool) {
+      case 1: LAQ_LAUNCH_POOL_SELECT_PAIR(1); break;
+      case 3: LAQ_LAUNCH_POOL_SELECT_PAIR(3); break;
+      case 5: LAQ_LAUNCH_POOL_SELECT_PAIR(5); break;
+      case 7: LAQ_LAUNCH_POOL_SELECT_PAIR(7); break;
+      default: LAQ_LAUNCH_POOL_SELECT_PAIR(0); break;
+    }
+#undef LAQ_LAUNCH_POOL_SELECT_PAIR
+    *launches += 1;
+    *done = true;
+    return LAQ_OK;
   }
   const size_t smem = (size_t)d.Ls * sizeof(float);
   if (smem > 200u * 1024u || d.U > 0x7fffffff) return LAQ_OK;  // the caller uses the two-kernel path

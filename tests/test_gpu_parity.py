@@ -697,6 +697,27 @@ def test_gather_of_more_units_than_one_grid_dimension_holds(laq):
     assert torch.equal(k_out, want_k) and torch.equal(v_out, want_v)
 
 
+def test_long_units_select_in_a_pair_of_thread_blocks(laq):
+    # 32768 < L - R <= 65536: two thread blocks share a unit's pooling and top-k
+    D, W, kernel = 128, 1, 7
+    # identical keys: every score ties; the kept set is [k/2, k/2 + Kb) and crosses the boundary
+    # between the two blocks, so the tie-break has to be split between them
+    for L, B in ((50000, 40000), (65536, 33000), (32800, 50)):
+        q = torch.randn((1, 2, 1, W, D), generator=torch.Generator().manual_seed(L)).to(torch.bfloat16)
+        k = torch.full((1, 2, 1, L, D), 0.25).to(torch.bfloat16)
+        v = torch.randn((1, 2, 1, L, D), generator=torch.Generator().manual_seed(L + 1)).to(torch.bfloat16)
+        out = run_evict(laq, q, k, v, W, kernel, B)
+        want = list(range(kernel // 2, kernel // 2 + B - W)) + list(range(L - W, L))
+        for b in range(2):
+            assert out["idx"][0, b, 0].cpu().tolist() == want, (L, B, b)
+            assert (bits(out["v_out"][0, b, 0]) == bits(v[0, b, 0])[np.array(want)]).all()
+    # random keys: scores against the oracle, selection bit-exact on the GPU's own scores
+    NL, Bt, Hq, Hkv, L, W, B = 1, 1, 4, 2, 60000, 4, 3000
+    q, k, v = rand_inputs(NL, Bt, Hq, Hkv, D, L, W, seed=75, kscale=1.5)
+    compare_all_units(laq, q, k, v, W, kernel, B)
+    compare_all_units(laq, q, k, v, W, 5, 40000, seq_lens=[45000], pool_mode=1)
+
+
 def test_config1_full_with_planted_key(laq):
     cfg = synth.CONFIGS[1]
     inp = synth.make_inputs(cfg, "cpu")
