@@ -122,3 +122,34 @@ def test_seq_lens_are_validated_on_host(binding):
     fake = ctypes.c_void_p(4096)
     assert binding.lib.laq_score(ctypes.byref(big), fake, fake, fake, fake, 1 << 40, None) == \
         binding.LAQ_ERR_UNSUPPORTED
+
+
+def test_layer_budget_pool_size_and_validation_on_the_host(binding):
+    p = binding.make_params(3, 2, 8, 2, 128, 1000, 4, 4, 7, 90)
+    assert binding.laq_layers_pool_entries(p, [90, 40, 64]) == 2 * 2 * (90 + 40 + 64)
+    assert binding.laq_layers_pool_entries(p, [80, 40, 64]) == 0      # p.budget must be the largest
+    assert binding.laq_layers_pool_entries(p, [90, 4, 64]) == 0       # a budget must exceed the tail
+    assert binding.laq_layers_pool_entries(p, [90, 1000, 64]) == 0    # and stay below the prompt length
+    p.group_mode = binding.LAQ_GROUP_PER_HEAD                         # one row of entries per query head
+    assert binding.laq_layers_pool_entries(p, [90, 40, 64]) == 2 * 8 * (90 + 40 + 64)
+    p.set_seq_lens([1000, 60])
+    assert binding.laq_layers_pool_entries(p, [90, 40, 64]) == 0      # a budget reaches a prompt's length
+
+
+def test_group_mode_and_streaming_arguments_are_checked_on_the_host(binding):
+    p = binding.make_params(1, 1, 8, 2, 128, 1000, 4, 4, 7, 90)
+    n = binding.laq_workspace_bytes(p)
+    p.group_mode = binding.LAQ_GROUP_MAX
+    assert binding.laq_workspace_bytes(p) > n          # per-head column sums need room
+    p.group_mode = 3
+    assert binding.laq_workspace_bytes(p) == 0
+    p.group_mode = binding.LAQ_GROUP_PER_HEAD
+    p.score_mode = binding.LAQ_SCORE_RAW
+    assert binding.laq_workspace_bytes(p) == 0         # unsupported together
+    p.group_mode, p.score_mode, p.reserved0 = 0, 0, 1
+    assert binding.laq_workspace_bytes(p) == 0
+    p.reserved0 = 0
+    for n_sink in (-1, 91):
+        st = binding.lib.laq_streaming_indices(ctypes.byref(p), n_sink, ctypes.c_void_p(16), None)
+        assert st == binding.LAQ_ERR_INVALID_ARG
+    assert binding.lib.laq_streaming_indices(ctypes.byref(p), 4, None, None) == binding.LAQ_ERR_INVALID_ARG
